@@ -1,0 +1,465 @@
+// Plain FFMA kernels: latent ingest, GroupNorm statistics, a tiled direct convolution with the
+// fused prologue/epilogue, a streaming-softmax attention, and weight repacking.  These run the
+// fp32 configuration end to end and serve as the on-GPU cross-check path of the bf16 one.
+#include <math.h>
+
+#include "vd_internal.h"
+
+namespace vd {
+
+namespace {
+
+template <typename T> __device__ __forceinline__ float ld_f(const T* p, size_t i);
+template <> __device__ __forceinline__ float ld_f<float>(const float* p, size_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ld_f<__nv_bfloat16>(const __nv_bfloat16* p, size_t i) {
+    return __bfloat162float(p[i]);
+}
+template <typename T> __device__ __forceinline__ void st_f(T* p, size_t i, float v);
+template <> __device__ __forceinline__ void st_f<float>(float* p, size_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void st_f<__nv_bfloat16>(__nv_bfloat16* p, size_t i, float v) {
+    p[i] = __float2bfloat16_rn(v);
+}
+__device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v)); }
+
+// ------------------------------------------------------------------------------------ ingest
+// Latents NCHW -> fp32 NHWC; optionally forms z = z_prev + lambda*v_prev first (Algorithm 2,
+// hit branch) and writes z and the new motion vector back in the latents' own layout/dtype.
+template <typename T>
+__global__ void ingest_kernel(IngestArgs a) {
+    const int64_t total = (int64_t)a.B * a.C * a.h * a.w;
+    const T* z = (const T*)a.z;
+    const T* vp = (const T*)a.v_prev;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        // i indexes the NCHW source
+        const int x = (int)(i % a.w);
+        const int y = (int)((i / a.w) % a.h);
+        const int c = (int)((i / ((int64_t)a.w * a.h)) % a.C);
+        const int n = (int)(i / ((int64_t)a.w * a.h * a.C));
+        float v = ld_f<T>(z, i);
+        if (vp) {
+            const float zp = v;
+            v = fmaf(a.lambda, ld_f<T>(vp, i), zp);
+            if (a.z_out) {               // what is decoded is the latent as stored in its own dtype
+                st_f<T>((T*)a.z_out, i, v);
+                v = ld_f<T>((const T*)a.z_out, i);
+            }
+            if (a.v_out) st_f<T>((T*)a.v_out, i, v - zp);
+        }
+        a.x[(((int64_t)n * a.h + y) * a.w + x) * a.C + c] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------ GroupNorm stats
+// Pass A: every block reduces a run of pixels of one sample to per-group (count, mean, M2).
+// A thread owns one 4-channel slot (inside one group, since C/G is a multiple of 4) and walks
+// down the pixels; sums are taken about the first value seen, so a large common offset does
+// not cancel; partial results are merged with the parallel-variance (Chan) update.
+struct Moments { float n, mean, m2; };
+__device__ __forceinline__ Moments merge(Moments a, Moments b) {
+    if (b.n == 0.f) return a;
+    if (a.n == 0.f) return b;
+    const float n = a.n + b.n;
+    const float d = b.mean - a.mean;
+    const float f = b.n / n;
+    Moments r;
+    r.n = n;
+    r.mean = fmaf(d, f, a.mean);
+    r.m2 = a.m2 + b.m2 + d * d * a.n * f;
+    return r;
+}
+
+template <typename T> __device__ __forceinline__ void load4(const T* p, float v[4]);
+template <> __device__ __forceinline__ void load4<float>(const float* p, float v[4]) {
+    const float4 t = __ldg((const float4*)p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, float v[4]) {
+    const uint2 t = __ldg((const uint2*)p);
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
+constexpr int kGnThreads = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kGnThreads) gn_partial_kernel(GnArgs a, int chunks, int pix_per_chunk) {
+    __shared__ Moments sm[kGnThreads];
+    const int n = blockIdx.y;
+    const int chunk = blockIdx.x;
+    const int slots = a.C / 4;                       // 4-channel slots per pixel (<= 128... or more: loop)
+    const int p0 = chunk * pix_per_chunk;
+    const int p1 = min(a.P, p0 + pix_per_chunk);
+    const T* x = (const T*)a.x + (size_t)n * a.P * a.C;
+    const int cpg = a.C / a.G;
+
+    // slot loop: when C/4 > blockDim (not the case for C <= 1024) a thread would own several slots
+    for (int slot0 = 0; slot0 < slots; slot0 += kGnThreads) {
+        const int lanes = min(slots - slot0, kGnThreads);       // threads across the channel axis
+        const int rows = kGnThreads / lanes;                    // pixels handled side by side
+        const int slot = slot0 + (threadIdx.x % lanes);
+        const int row = threadIdx.x / lanes;
+        Moments m = {0.f, 0.f, 0.f};
+        if (row < rows && p0 + row < p1) {
+            float v[4];
+            load4<T>(x + (size_t)(p0 + row) * a.C + slot * 4, v);
+            const float k = v[0];
+            float s = 0.f, ss = 0.f, cnt = 0.f;
+            int p = p0 + row;
+            for (; p + 3 * rows < p1; p += 4 * rows) {
+                float u[4][4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) load4<T>(x + (size_t)(p + j * rows) * a.C + slot * 4, u[j]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float d = u[j][e] - k;
+                        s += d;
+                        ss = fmaf(d, d, ss);
+                    }
+                cnt += 16.f;
+            }
+            for (; p < p1; p += rows) {
+                load4<T>(x + (size_t)p * a.C + slot * 4, v);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float d = v[e] - k;
+                    s += d;
+                    ss = fmaf(d, d, ss);
+                }
+                cnt += 4.f;
+            }
+            const float md = s / cnt;
+            m.n = cnt;
+            m.mean = k + md;
+            m.m2 = fmaxf(ss - s * md, 0.f);
+        }
+        sm[threadIdx.x] = m;
+        __syncthreads();
+        // one thread per group present in this slot window gathers its members
+        const int g_lo = (slot0 * 4) / cpg;
+        const int g_hi = ((slot0 + lanes) * 4 - 1) / cpg;
+        const int g = g_lo + threadIdx.x;
+        if (g <= g_hi) {
+            const int s_lo = max(g * cpg / 4 - slot0, 0);
+            const int s_hi = min((g + 1) * cpg / 4 - slot0, lanes);
+            Moments acc = {0.f, 0.f, 0.f};
+            for (int r = 0; r < rows; ++r)
+                for (int sl = s_lo; sl < s_hi; ++sl) acc = merge(acc, sm[r * lanes + sl]);
+            float* out = a.partial + (((size_t)n * kGnMaxChunks + chunk) * a.G + g) * 4;
+            if (slot0 > 0 && (slot0 * 4) % cpg != 0 && g == g_lo) {
+                // group straddles two slot windows: fold into what the previous window wrote
+                Moments prev = {out[0], out[1], out[2]};
+                acc = merge(prev, acc);
+            }
+            out[0] = acc.n; out[1] = acc.mean; out[2] = acc.m2;
+        }
+        __syncthreads();
+    }
+}
+
+// Pass B: one warp per (sample, group) merges the chunk partials (lanes stride over the chunks,
+// then a shuffle tree), and folds the statistics with the affine parameters into per-(sample,
+// channel) scale and shift.
+__global__ void gn_finalize_kernel(GnArgs a, int chunks) {
+    const int n = blockIdx.x;
+    const int cpg = a.C / a.G;
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32, nwarps = blockDim.x / 32;
+    for (int g = warp; g < a.G; g += nwarps) {
+        Moments m = {0.f, 0.f, 0.f};
+        for (int k = lane; k < chunks; k += 32) {
+            const float4 p = *(const float4*)(a.partial + (((size_t)n * kGnMaxChunks + k) * a.G + g) * 4);
+            m = merge(m, Moments{p.x, p.y, p.z});
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            Moments o;
+            o.n = __shfl_xor_sync(0xffffffffu, m.n, d);
+            o.mean = __shfl_xor_sync(0xffffffffu, m.mean, d);
+            o.m2 = __shfl_xor_sync(0xffffffffu, m.m2, d);
+            m = merge(m, o);
+        }
+        const float cnt = __shfl_sync(0xffffffffu, m.n, 0);
+        const float mean = __shfl_sync(0xffffffffu, m.mean, 0);
+        const float m2 = __shfl_sync(0xffffffffu, m.m2, 0);
+        const float rstd = (float)(1.0 / sqrt((double)m2 / (double)cnt + (double)a.eps));
+        for (int cc = lane; cc < cpg; cc += 32) {
+            const int c = g * cpg + cc;
+            const float sc = a.gamma[c] * rstd;
+            a.scale[(size_t)n * a.C + c] = sc;
+            a.shift[(size_t)n * a.C + c] = a.beta[c] - mean * sc;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------- direct conv
+// Block = TH x TW output pixels x CT output channels; input channels are consumed KC at a time
+// through shared memory (the transformed input tile with its halo, and the weight slice).
+constexpr int KC = 8;
+
+template <typename TIn, typename TOut, int TH, int TW, int PPT, int CPT, int CGROUPS>
+__global__ void __launch_bounds__((TH * TW / PPT) * CGROUPS) conv_simt_kernel(ConvArgs a) {
+    constexpr int NPG = TH * TW / PPT;
+    constexpr int CT = CPT * CGROUPS;
+    constexpr int NT = NPG * CGROUPS;
+    constexpr int PW = TW + 2, PH = TH + 2, NPIX = PW * PH;
+    __shared__ float s_in[KC][NPIX + 1];
+    __shared__ float s_w[9][KC][CT];
+
+    const int tiles_x = (a.W + TW - 1) / TW;
+    const int tx0 = (blockIdx.x % tiles_x) * TW;
+    const int ty0 = (blockIdx.x / tiles_x) * TH;
+    const int ct0 = blockIdx.y * CT;
+    const int b = blockIdx.z;
+    const int tid = threadIdx.x;
+    const int pg = tid % NPG, cg = tid / NPG;
+    const int ly = (pg * PPT) / TW, lx = (pg * PPT) % TW;
+    const int taps = a.ksize * a.ksize;
+    const int up = a.upsample ? 1 : 0;
+
+    float acc[PPT][CPT];
+#pragma unroll
+    for (int p = 0; p < PPT; ++p)
+#pragma unroll
+        for (int q = 0; q < CPT; ++q) acc[p][q] = 0.f;
+
+    const TIn* x = (const TIn*)a.x + (size_t)b * a.Hs * a.Ws * a.Cin;
+    const float* wp = (const float*)a.w;
+
+    for (int c0 = 0; c0 < a.Cin; c0 += KC) {
+        for (int idx = tid; idx < NPIX * KC; idx += NT) {
+            const int c = idx % KC, pix = idx / KC;
+            const int oy = ty0 + pix / PW - 1, ox = tx0 + pix % PW - 1;
+            float v = 0.f;
+            if (oy >= 0 && oy < a.H && ox >= 0 && ox < a.W && c0 + c < a.Cin) {
+                v = ld_f<TIn>(x, ((size_t)(oy >> up) * a.Ws + (ox >> up)) * a.Cin + c0 + c);
+                if (a.scale) v = fmaf(v, a.scale[(size_t)b * a.Cin + c0 + c], a.shift[(size_t)b * a.Cin + c0 + c]);
+                if (a.silu) v = silu_f(v);
+                if (a.bf16_operands) v = round_bf16(v);
+            }
+            s_in[c][pix] = v;
+        }
+        for (int idx = tid; idx < taps * KC * CT; idx += NT) {
+            const int ct = idx % CT, c = (idx / CT) % KC, tap = idx / (CT * KC);
+            float v = 0.f;
+            if (c0 + c < a.Cin && ct0 + ct < a.Cout) v = wp[((size_t)tap * a.Cin + c0 + c) * a.Cout + ct0 + ct];
+            s_w[tap][c][ct] = v;
+        }
+        __syncthreads();
+        for (int tap = 0; tap < taps; ++tap) {
+            const int dy = a.ksize == 3 ? tap / 3 : 1, dx = a.ksize == 3 ? tap % 3 : 1;
+            const int base = (ly + dy) * PW + lx + dx;
+#pragma unroll
+            for (int c = 0; c < KC; ++c) {
+                float iv[PPT], wv[CPT];
+#pragma unroll
+                for (int p = 0; p < PPT; ++p) iv[p] = s_in[c][base + p];
+#pragma unroll
+                for (int q = 0; q < CPT; ++q) wv[q] = s_w[tap][c][cg * CPT + q];
+#pragma unroll
+                for (int p = 0; p < PPT; ++p)
+#pragma unroll
+                    for (int q = 0; q < CPT; ++q) acc[p][q] = fmaf(iv[p], wv[q], acc[p][q]);
+            }
+        }
+        __syncthreads();
+    }
+
+    TOut* y = (TOut*)a.y;
+#pragma unroll
+    for (int p = 0; p < PPT; ++p) {
+        const int oy = ty0 + ly, ox = tx0 + lx + p;
+        if (oy >= a.H || ox >= a.W) continue;
+#pragma unroll
+        for (int q = 0; q < CPT; ++q) {
+            const int co = ct0 + cg * CPT + q;
+            if (co >= a.Cout) continue;
+            float v = acc[p][q];
+            if (a.bias) v += a.bias[co];
+            const size_t nhwc = (((size_t)b * a.H + oy) * a.W + ox) * a.Cout + co;
+            if (a.residual) v += a.residual[nhwc];
+            const size_t o = a.out_nchw ? (((size_t)b * a.Cout + co) * a.H + oy) * a.W + ox : nhwc;
+            st_f<TOut>(y, o, v);
+        }
+    }
+}
+
+template <typename TIn, typename TOut>
+cudaError_t conv_simt_dispatch(const ConvArgs& a, cudaStream_t s) {
+    if (a.Cout <= 8) {
+        constexpr int TH = 16, TW = 16, CT = 4;
+        dim3 grid(((a.W + TW - 1) / TW) * ((a.H + TH - 1) / TH), (a.Cout + CT - 1) / CT, a.B);
+        conv_simt_kernel<TIn, TOut, TH, TW, 1, 4, 1><<<grid, 256, 0, s>>>(a);
+    } else {
+        constexpr int TH = 8, TW = 8, CT = 64;
+        dim3 grid(((a.W + TW - 1) / TW) * ((a.H + TH - 1) / TH), (a.Cout + CT - 1) / CT, a.B);
+        conv_simt_kernel<TIn, TOut, TH, TW, 4, 4, 16><<<grid, 256, 0, s>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------------------------------------- attention
+// One warp per query, eight queries per block sharing 32-key K/V tiles in shared memory;
+// running maximum / running sum softmax, all in fp32.
+constexpr int kAttnQ = 8, kAttnKeys = 32;
+
+template <typename T>
+__global__ void __launch_bounds__(kAttnQ * 32) attn_simt_kernel(AttnArgs a) {
+    extern __shared__ float smem[];
+    const int C = a.C;
+    float* s_q = smem;                               // [kAttnQ][C]
+    float* s_k = s_q + kAttnQ * C;                   // [kAttnKeys][C+1]
+    float* s_v = s_k + kAttnKeys * (C + 1);          // [kAttnKeys][C]
+    const int b = blockIdx.y;
+    const int q0 = blockIdx.x * kAttnQ;
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const T* q = (const T*)a.q + (size_t)b * a.T * a.ld_qkv;
+    const T* k = (const T*)a.k + (size_t)b * a.T * a.ld_qkv;
+    const T* v = (const T*)a.v + (size_t)b * a.T * a.ld_qkv;
+    T* o = (T*)a.o + (size_t)b * a.T * a.ld_o;
+
+    for (int idx = threadIdx.x; idx < kAttnQ * C; idx += blockDim.x) {
+        const int qi = idx / C, c = idx % C;
+        s_q[idx] = (q0 + qi < a.T) ? ld_f<T>(q, (size_t)(q0 + qi) * a.ld_qkv + c) : 0.f;
+    }
+    const int nacc = C / 32;                          // channels per lane (C multiple of 32, <= 512)
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    float m = -INFINITY, l = 0.f;
+
+    for (int k0 = 0; k0 < a.T; k0 += kAttnKeys) {
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < kAttnKeys * C; idx += blockDim.x) {
+            const int ki = idx / C, c = idx % C;
+            const bool ok = k0 + ki < a.T;
+            s_k[ki * (C + 1) + c] = ok ? ld_f<T>(k, (size_t)(k0 + ki) * a.ld_qkv + c) : 0.f;
+            s_v[ki * C + c] = ok ? ld_f<T>(v, (size_t)(k0 + ki) * a.ld_qkv + c) : 0.f;
+        }
+        __syncthreads();
+        float sc = 0.f;
+        const float* qr = s_q + warp * C;
+        const float* kr = s_k + lane * (C + 1);
+        for (int c = 0; c < C; ++c) sc = fmaf(qr[c], kr[c], sc);
+        sc = (k0 + lane < a.T) ? sc * a.scale : -INFINITY;
+        float tmax = sc;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, d));
+        const float m_new = fmaxf(m, tmax);
+        const float corr = expf(m - m_new);           // m = -inf at the first tile: exp(-inf) = 0
+        const float p = expf(sc - m_new);
+        float psum = p;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, d);
+        l = l * corr + psum;
+        m = m_new;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] *= corr;
+        for (int ki = 0; ki < kAttnKeys; ++ki) {
+            const float pk = __shfl_sync(0xffffffffu, p, ki);
+            const float* vr = s_v + ki * C + lane;
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (i < nacc) acc[i] = fmaf(pk, vr[i * 32], acc[i]);
+        }
+    }
+    if (q0 + warp < a.T) {
+        const float inv = 1.f / l;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (i < nacc) st_f<T>(o, (size_t)(q0 + warp) * a.ld_o + lane + i * 32, acc[i] * inv);
+    }
+}
+
+// ------------------------------------------------------------------------------------ repack
+template <typename T>
+__global__ void pack_weight_simt_kernel(const T* w, float* packed, int Cout, int Cin, int taps, int cout_total,
+                                        int cout_offset) {
+    const int64_t total = (int64_t)Cout * Cin * taps;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int tap = (int)(i % taps);
+        const int c = (int)((i / taps) % Cin);
+        const int o = (int)(i / ((int64_t)taps * Cin));
+        packed[((size_t)tap * Cin + c) * cout_total + cout_offset + o] = ld_f<T>(w, i);
+    }
+}
+
+template <typename T>
+__global__ void to_f32_kernel(const T* src, float* dst, int64_t n) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = ld_f<T>(src, i);
+}
+
+int grid_for(int64_t n, int threads) {
+    int64_t g = (n + threads - 1) / threads;
+    if (g < 1) g = 1;
+    if (g > 148 * 16) g = 148 * 16;
+    return (int)g;
+}
+
+}  // namespace
+
+cudaError_t launch_ingest(const IngestArgs& a, cudaStream_t s) {
+    const int64_t n = (int64_t)a.B * a.C * a.h * a.w;
+    if (a.dtype == VD_BF16) ingest_kernel<__nv_bfloat16><<<grid_for(n, 256), 256, 0, s>>>(a);
+    else ingest_kernel<float><<<grid_for(n, 256), 256, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s) {
+    // chunks per sample depend on the sample size only (so a frame's statistics, and with them
+    // the frame, do not depend on the batch it is decoded in): at least 32 pixels per chunk
+    int ppc = max(32, (a.P + kGnMaxChunks - 1) / kGnMaxChunks);
+    int chunks = (a.P + ppc - 1) / ppc;
+    dim3 grid(chunks, a.B);
+    if (a.dtype == VD_BF16) gn_partial_kernel<__nv_bfloat16><<<grid, kGnThreads, 0, s>>>(a, chunks, ppc);
+    else gn_partial_kernel<float><<<grid, kGnThreads, 0, s>>>(a, chunks, ppc);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    gn_finalize_kernel<<<a.B, 256, 0, s>>>(a, chunks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_conv_simt(const ConvArgs& a, cudaStream_t s) {
+    const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
+    if (ib && ob) return conv_simt_dispatch<__nv_bfloat16, __nv_bfloat16>(a, s);
+    if (ib && !ob) return conv_simt_dispatch<__nv_bfloat16, float>(a, s);
+    if (!ib && ob) return conv_simt_dispatch<float, __nv_bfloat16>(a, s);
+    return conv_simt_dispatch<float, float>(a, s);
+}
+
+cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s) {
+    if (a.C % 32 != 0 || a.C > 512) return cudaErrorInvalidValue;
+    const size_t smem = sizeof(float) * ((size_t)kAttnQ * a.C + (size_t)kAttnKeys * (a.C + 1) + (size_t)kAttnKeys * a.C);
+    dim3 grid((a.T + kAttnQ - 1) / kAttnQ, a.B);
+    cudaError_t e;
+    if (a.dtype == VD_BF16) {
+        e = cudaFuncSetAttribute(attn_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attn_simt_kernel<__nv_bfloat16><<<grid, kAttnQ * 32, smem, s>>>(a);
+    } else {
+        e = cudaFuncSetAttribute(attn_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attn_simt_kernel<float><<<grid, kAttnQ * 32, smem, s>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack_weight_simt(const void* w, int w_dtype, float* packed, int Cout, int Cin, int taps,
+                                    int cout_total, int cout_offset, cudaStream_t s) {
+    const int64_t n = (int64_t)Cout * Cin * taps;
+    if (w_dtype == VD_BF16)
+        pack_weight_simt_kernel<__nv_bfloat16><<<grid_for(n, 256), 256, 0, s>>>((const __nv_bfloat16*)w, packed, Cout, Cin, taps, cout_total, cout_offset);
+    else
+        pack_weight_simt_kernel<float><<<grid_for(n, 256), 256, 0, s>>>((const float*)w, packed, Cout, Cin, taps, cout_total, cout_offset);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cudaStream_t s) {
+    if (dtype == VD_BF16) to_f32_kernel<__nv_bfloat16><<<grid_for(n, 256), 256, 0, s>>>((const __nv_bfloat16*)src, dst, n);
+    else to_f32_kernel<float><<<grid_for(n, 256), 256, 0, s>>>((const float*)src, dst, n);
+    return cudaGetLastError();
+}
+
+}  // namespace vd

@@ -1,0 +1,688 @@
+// C ABI of libvd.so: argument validation, the per-configuration launch plan (layer list ->
+// kernel launches and workspace offsets), weight repacking at create time, and the decode loop.
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "vd_internal.h"
+
+using namespace vd;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+struct Step {
+    vd_step_info info;
+    int kind;
+    bool use_tc;
+    ConvArgs conv;
+    GnArgs gn;
+    AttnArgs attn;
+    IngestArgs ing;
+    ConvTcPlan tc;
+    // batch-dependent pointers are rebased per call: strides per frame
+    bool has_residual;
+};
+
+struct WeightJob {           // repack work done once in vd_create
+    std::string name;        // source tensor
+    int kind;                // 0 conv weight (packed), 1 vector -> fp32
+    bool tc;
+    int Cout, Cin, taps;
+    int cout_total, cout_offset;
+    size_t dst_off;
+};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+int elt(int dtype) { return dtype == VD_BF16 ? 2 : 4; }
+
+}  // namespace
+
+struct vd_handle_s {
+    vd_config cfg;
+    char* ws = nullptr;
+    size_t ws_bytes = 0;
+    std::vector<Step> steps;
+    std::vector<WeightJob> jobs;
+    std::string err;
+    int stop_after = -1;
+    size_t status_off = 0, lat_stage_off = 0, frm_stage_off = 0;
+    size_t total = 0;
+};
+
+namespace {
+
+// Walks the layer list of a layout and lays out workspace + steps.  With base == nullptr only
+// sizes/offsets are computed (all pointers are offsets from 0).
+class Planner {
+  public:
+    Planner(vd_handle_s* h, char* base) : h_(h), base_(base), cfg_(h->cfg) {}
+
+    size_t alloc(size_t bytes) {
+        const size_t off = align_up(cur_, 256);
+        cur_ = off + bytes;
+        return off;
+    }
+    template <typename T> T* ptr(size_t off) const { return (T*)(base_ + off); }
+
+    bool bf16() const { return cfg_.dtype == VD_BF16; }
+    int act_dtype() const { return bf16() ? VD_BF16 : VD_F32; }   // intra-block tensors
+
+    struct ConvW { size_t w_off, b_off; bool tc; };
+
+    // registers the repack of a conv weight (possibly a stack of several source tensors along Cout)
+    ConvW conv_weight(const std::vector<std::string>& names, int Cout_each, int Cin, int taps, bool tc) {
+        const int Cout = Cout_each * (int)names.size();
+        ConvW r;
+        r.tc = tc;
+        const size_t wbytes = tc ? conv_tc_packed_bytes(Cout, Cin, taps) : (size_t)taps * Cin * Cout * 4;
+        r.w_off = alloc(wbytes);
+        r.b_off = alloc((size_t)Cout * 4);
+        for (size_t i = 0; i < names.size(); ++i) {
+            h_->jobs.push_back({names[i] + ".weight", 0, tc, Cout_each, Cin, taps, Cout, (int)i * Cout_each, r.w_off});
+            h_->jobs.push_back({names[i] + ".bias", 1, false, Cout_each, 0, 0, 0, 0, r.b_off + (size_t)i * Cout_each * 4});
+        }
+        return r;
+    }
+    void norm_weight(const std::string& name, int C, size_t& g_off, size_t& b_off) {
+        g_off = alloc((size_t)C * 4);
+        b_off = alloc((size_t)C * 4);
+        h_->jobs.push_back({name + ".weight", 1, false, C, 0, 0, 0, 0, g_off});
+        h_->jobs.push_back({name + ".bias", 1, false, C, 0, 0, 0, 0, b_off});
+    }
+
+    void add_gn(const std::string& name, size_t x_off, int dtype, int H, int W, int C, const std::string& wname) {
+        Step s{};
+        s.kind = VD_STEP_GN_STATS;
+        size_t g_off, b_off;
+        norm_weight(wname, C, g_off, b_off);
+        s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
+                      ptr<float>(b_off), ptr<float>(scale_off_), ptr<float>(shift_off_), ptr<float>(partial_off_)};
+        fill_info(s, name, 0, C, C, 0, 0, H, W, C, VD_F32, 0, -1);
+        s.info.launches = 2;
+        s.info.bytes_per_frame = (double)H * W * C * elt(dtype);
+        h_->steps.push_back(s);
+    }
+
+    // conv step; x at source resolution Hs x Ws
+    void add_conv(const std::string& name, const std::vector<std::string>& wnames, int Cout_each, size_t x_off,
+                  int in_dtype, int Hs, int Ws, int Cin, int ksize, bool upsample, bool prologue, bool silu,
+                  long residual_off, size_t y_off, int out_dtype, bool out_nchw, bool y_is_frames) {
+        Step s{};
+        s.kind = VD_STEP_CONV;
+        const int Cout = Cout_each * (int)wnames.size();
+        const int H = upsample ? 2 * Hs : Hs, W = upsample ? 2 * Ws : Ws;
+        ConvArgs a{};
+        a.x = ptr<void>(x_off);
+        a.scale = prologue ? ptr<float>(scale_off_) : nullptr;
+        a.shift = prologue ? ptr<float>(shift_off_) : nullptr;
+        a.residual = residual_off >= 0 ? ptr<float>((size_t)residual_off) : nullptr;
+        a.y = y_is_frames ? nullptr : ptr<void>(y_off);
+        a.B = 0; a.Hs = Hs; a.Ws = Ws; a.H = H; a.W = W;
+        a.Cin = Cin; a.Cout = Cout; a.ksize = ksize; a.upsample = upsample; a.silu = silu;
+        a.in_dtype = in_dtype; a.out_dtype = out_dtype; a.out_nchw = out_nchw; a.bf16_operands = bf16();
+        ConvArgs probe = a;
+        probe.B = 1;
+        const bool tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && conv_tc_supported(probe);
+        ConvW cw = conv_weight(wnames, Cout_each, Cin, ksize * ksize, tc);
+        a.w = ptr<void>(cw.w_off);
+        a.bias = ptr<float>(cw.b_off);
+        s.conv = a;
+        s.use_tc = tc;
+        s.has_residual = residual_off >= 0;
+        fill_info(s, name, tc, Cin, Cout, ksize, upsample, H, W, Cout, out_dtype, out_nchw, y_is_frames ? -1 : (long)y_off);
+        const double P = (double)H * W;
+        s.info.flops_per_frame = 2.0 * ksize * ksize * Cin * (double)Cout * P;
+        s.info.bytes_per_frame = (double)Hs * Ws * Cin * elt(in_dtype) + P * Cout * elt(out_dtype) +
+                                 (residual_off >= 0 ? P * Cout * 4.0 : 0.0);
+        s.info.weight_bytes = (double)ksize * ksize * Cin * Cout * elt(cfg_.dtype);
+        h_->steps.push_back(s);
+    }
+
+    void fill_info(Step& s, const std::string& name, int impl, int cin, int cout, int ksize, int up, int H, int W,
+                   int oc, int odt, int nchw, long off) {
+        memset(&s.info, 0, sizeof(s.info));
+        snprintf(s.info.name, sizeof(s.info.name), "%s", name.c_str());
+        s.info.kind = s.kind; s.info.impl = impl; s.info.launches = 1;
+        s.info.c_in = cin; s.info.c_out = cout; s.info.ksize = ksize; s.info.upsample = up;
+        s.info.out_h = H; s.info.out_w = W; s.info.out_channels = oc; s.info.out_dtype = odt;
+        s.info.out_nchw = nchw; s.info.out_offset = off;
+    }
+
+    // x -> shortcut(x) + conv2(silu(gn2(conv1(silu(gn1(x))))))
+    void resblock(const std::string& p, int Cin, int Cout, int H, int W) {
+        const size_t x = xs_[cur_x_], y = xs_[cur_x_ ^ 1];
+        add_gn(p + ".norm1", x, VD_F32, H, W, Cin, p + ".norm1");
+        add_conv(p + ".conv1", {p + ".conv1"}, Cout, x, VD_F32, H, W, Cin, 3, false, true, true, -1, hbuf_, act_dtype(),
+                 false, false);
+        add_gn(p + ".norm2", hbuf_, act_dtype(), H, W, Cout, p + ".norm2");
+        long res = (long)x;
+        if (Cin != Cout) {
+            add_conv(p + ".shortcut", {p + ".shortcut"}, Cout, x, VD_F32, H, W, Cin, 1, false, false, false, -1, sbuf_,
+                     VD_F32, false, false);
+            res = (long)sbuf_;
+        }
+        add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, res, y,
+                 VD_F32, false, false);
+        cur_x_ ^= 1;
+    }
+
+    void attention(const std::string& p, int C, int H, int W) {
+        const size_t x = xs_[cur_x_], y = xs_[cur_x_ ^ 1];
+        add_gn(p + ".norm", x, VD_F32, H, W, C, p + ".norm");
+        add_conv(p + ".qkv", {p + ".q", p + ".k", p + ".v"}, C, x, VD_F32, H, W, C, 1, false, true, false, -1, qkv_,
+                 act_dtype(), false, false);
+        Step s{};
+        s.kind = VD_STEP_ATTENTION;
+        const int es = elt(act_dtype());
+        s.attn = AttnArgs{ptr<void>(qkv_), ptr<void>(qkv_ + (size_t)C * es), ptr<void>(qkv_ + (size_t)2 * C * es),
+                          ptr<void>(attno_), act_dtype(), 0, H * W, C, 3 * C, C, 1.0f / sqrtf((float)C)};
+        s.use_tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && attn_tc_supported(s.attn);
+        fill_info(s, p + ".core", s.use_tc, C, C, 0, 0, H, W, C, act_dtype(), 0, (long)attno_);
+        const double T = (double)H * W;
+        s.info.flops_per_frame = 4.0 * T * T * C;
+        s.info.bytes_per_frame = 4.0 * T * C * es;
+        h_->steps.push_back(s);
+        add_conv(p + ".o", {p + ".o"}, C, attno_, act_dtype(), H, W, C, 1, false, false, false, (long)x, y, VD_F32,
+                 false, false);
+        cur_x_ ^= 1;
+    }
+
+    void upconv(const std::string& p, int Cin, int Cout, int Hs, int Ws) {
+        add_conv(p, {p}, Cout, xs_[cur_x_], VD_F32, Hs, Ws, Cin, 3, true, false, false, -1, xs_[cur_x_ ^ 1], VD_F32,
+                 false, false);
+        cur_x_ ^= 1;
+    }
+
+    vd_status plan() {
+        const int h = cfg_.latent_h, w = cfg_.latent_w, B = cfg_.max_batch;
+        const int lc = cfg_.latent_channels;
+        const size_t P0 = (size_t)h * w;
+        // ---- sizes of the shared activation buffers (per frame), by walking the widths
+        size_t max_x = 0, max_h = 0, max_s = 0, max_c = 0, qkv = 0, ao = 0;
+        if (cfg_.arch == VD_ARCH_SDVAE) {
+            const int ch[4] = {512, 512, 256, 128};
+            size_t P = P0;
+            max_x = P * 512;
+            max_h = P * 512;
+            max_c = 512;
+            int prev = 512;
+            for (int i = 0; i < 4; ++i) {
+                max_x = std::max(max_x, P * (size_t)std::max(prev, ch[i]));
+                max_h = std::max(max_h, P * (size_t)ch[i]);
+                if (prev != ch[i]) max_s = std::max(max_s, P * (size_t)ch[i]);
+                prev = ch[i];
+                if (i < 3) { P *= 4; max_x = std::max(max_x, P * (size_t)ch[i]); }
+            }
+            qkv = P0 * 1536;
+            ao = P0 * 512;
+        } else {
+            const int st[3][2] = {{64, 64}, {64, 32}, {32, 32}};
+            size_t P = P0;
+            max_x = P * 64; max_h = P * 64; max_c = 64;
+            for (int i = 0; i < 3; ++i) {
+                P *= 4;
+                max_x = std::max(max_x, P * (size_t)st[i][1]);
+                max_h = std::max(max_h, P * (size_t)st[i][1]);
+            }
+        }
+        const int ae = elt(act_dtype());
+        h_->status_off = alloc(256);
+        scale_off_ = alloc((size_t)B * max_c * 4);
+        shift_off_ = alloc((size_t)B * max_c * 4);
+        partial_off_ = alloc(vd_gn_scratch_bytes(B, cfg_.norm_groups));
+        zbuf_ = alloc((size_t)B * P0 * lc * 4);
+        xs_[0] = alloc((size_t)B * max_x * 4);
+        xs_[1] = alloc((size_t)B * max_x * 4);
+        hbuf_ = alloc((size_t)B * max_h * ae);
+        sbuf_ = max_s ? alloc((size_t)B * max_s * 4) : 0;
+        qkv_ = qkv ? alloc((size_t)B * qkv * ae) : 0;
+        attno_ = ao ? alloc((size_t)B * ao * ae) : 0;
+        h_->lat_stage_off = alloc((size_t)B * P0 * lc * elt(cfg_.dtype));
+        h_->frm_stage_off = alloc((size_t)B * P0 * 64 * cfg_.out_channels * elt(cfg_.dtype));
+
+        // ---- steps
+        {
+            Step s{};
+            s.kind = VD_STEP_INGEST;
+            s.ing = IngestArgs{nullptr, nullptr, nullptr, nullptr, 0.f, ptr<float>(zbuf_), cfg_.dtype, 0, lc, h, w};
+            fill_info(s, "ingest", 0, lc, lc, 0, 0, h, w, lc, VD_F32, 0, (long)zbuf_);
+            s.info.bytes_per_frame = (double)P0 * lc * (elt(cfg_.dtype) + 4);
+            h_->steps.push_back(s);
+        }
+        cur_x_ = 0;
+        int H = h, W = w;
+        if (cfg_.arch == VD_ARCH_SDVAE) {
+            add_conv("conv_in", {"conv_in"}, 512, zbuf_, VD_F32, H, W, lc, 3, false, false, false, -1, xs_[0], VD_F32, false, false);
+            resblock("mid.res0", 512, 512, H, W);
+            attention("mid.attn", 512, H, W);
+            resblock("mid.res1", 512, 512, H, W);
+            const int ch[4] = {512, 512, 256, 128};
+            int prev = 512;
+            for (int i = 0; i < 4; ++i) {
+                for (int j = 0; j < 3; ++j) {
+                    char nm[32];
+                    snprintf(nm, sizeof(nm), "up%d.res%d", i, j);
+                    resblock(nm, j == 0 ? prev : ch[i], ch[i], H, W);
+                }
+                prev = ch[i];
+                if (i < 3) {
+                    char nm[32];
+                    snprintf(nm, sizeof(nm), "up%d.upconv", i);
+                    upconv(nm, ch[i], ch[i], H, W);
+                    H *= 2; W *= 2;
+                }
+            }
+            head(prev, H, W);
+        } else {
+            add_conv("conv_in", {"conv_in"}, 64, zbuf_, VD_F32, H, W, lc, 3, false, false, false, -1, xs_[0], VD_F32, false, false);
+            resblock("mid.res0", 64, 64, H, W);
+            const int st[3][2] = {{64, 64}, {64, 32}, {32, 32}};
+            for (int i = 0; i < 3; ++i) {
+                char nm[32];
+                snprintf(nm, sizeof(nm), "up%d.upconv", i);
+                upconv(nm, st[i][0], st[i][1], H, W);
+                H *= 2; W *= 2;
+                snprintf(nm, sizeof(nm), "up%d.res0", i);
+                resblock(nm, st[i][1], st[i][1], H, W);
+            }
+            head(32, H, W);
+        }
+        h_->total = align_up(cur_, 256);
+        return VD_OK;
+    }
+
+    void head(int C, int H, int W) {
+        add_gn("norm_out", xs_[cur_x_], VD_F32, H, W, C, "norm_out");
+        add_conv("conv_out", {"conv_out"}, cfg_.out_channels, xs_[cur_x_], VD_F32, H, W, C, 3, false, true, true, -1, 0,
+                 cfg_.dtype, true, true);
+    }
+
+  private:
+    vd_handle_s* h_;
+    char* base_;
+    const vd_config& cfg_;
+    size_t cur_ = 0;
+    size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, sbuf_ = 0, qkv_ = 0, attno_ = 0;
+    size_t xs_[2] = {0, 0};
+    int cur_x_ = 0;
+};
+
+vd_status validate_cfg(const vd_config* cfg, std::string& err) {
+    if (!cfg) { err = "config is NULL"; return VD_ERR_INVALID_ARG; }
+    if (cfg->struct_size != sizeof(vd_config)) { err = "config.struct_size does not match this library"; return VD_ERR_INVALID_ARG; }
+    if (cfg->arch != VD_ARCH_TINY && cfg->arch != VD_ARCH_SDVAE) { err = "unknown arch"; return VD_ERR_INVALID_ARG; }
+    if (cfg->dtype != VD_F32 && cfg->dtype != VD_BF16) { err = "unknown dtype"; return VD_ERR_INVALID_ARG; }
+    if (cfg->latent_channels != 4 || cfg->out_channels != 3) { err = "latent_channels must be 4 and out_channels 3"; return VD_ERR_UNSUPPORTED; }
+    if (cfg->latent_h < 1 || cfg->latent_w < 1 || cfg->latent_h > 4096 || cfg->latent_w > 4096) { err = "latent size out of range"; return VD_ERR_INVALID_ARG; }
+    if (cfg->max_batch < 1 || cfg->max_batch > 1024) { err = "max_batch out of range"; return VD_ERR_INVALID_ARG; }
+    const int cmin = cfg->arch == VD_ARCH_SDVAE ? 128 : 32;
+    if (cfg->norm_groups < 1 || cmin % cfg->norm_groups != 0 || (cmin / cfg->norm_groups) % 4 != 0) {
+        err = "norm_groups must divide every width into groups of a multiple of 4 channels";
+        return VD_ERR_INVALID_ARG;
+    }
+    if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~VD_FLAG_FORCE_SIMT) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    return VD_OK;
+}
+
+vd_status fail(vd_handle h, vd_status st, const std::string& msg) {
+    if (h) h->err = msg;
+    g_last_error = msg;
+    return st;
+}
+vd_status cuda_fail(vd_handle h, cudaError_t e, const char* where) {
+    return fail(h, VD_ERR_CUDA, std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+const vd_tensor* find_tensor(const vd_tensor* t, int n, const std::string& name) {
+    for (int i = 0; i < n; ++i)
+        if (t[i].name && name == t[i].name) return &t[i];
+    return nullptr;
+}
+
+cudaError_t launch_step(const vd_handle_s* h, const Step& st, int B, const void* latents, const void* v_prev,
+                        float lambda, void* z_out, void* v_out, void* frames, cudaStream_t s) {
+    unsigned int* status = (unsigned int*)(h->ws + h->status_off);
+    switch (st.kind) {
+        case VD_STEP_INGEST: {
+            IngestArgs a = st.ing;
+            a.B = B; a.z = latents; a.v_prev = v_prev; a.lambda = lambda; a.z_out = z_out; a.v_out = v_out;
+            return launch_ingest(a, s);
+        }
+        case VD_STEP_GN_STATS: {
+            GnArgs a = st.gn;
+            a.B = B;
+            return launch_gn_stats(a, s);
+        }
+        case VD_STEP_CONV: {
+            ConvArgs a = st.conv;
+            a.B = B;
+            if (!a.y) a.y = frames;
+            return st.use_tc ? launch_conv_tc(a, st.tc, status, s) : launch_conv_simt(a, s);
+        }
+        case VD_STEP_ATTENTION: {
+            AttnArgs a = st.attn;
+            a.B = B;
+            return st.use_tc ? launch_attn_tc(a, status, s) : launch_attn_simt(a, s);
+        }
+    }
+    return cudaErrorInvalidValue;
+}
+
+vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, float lambda, void* z_out, void* v_out,
+                      void* frames, int32_t batch, void* stream, float* ms, int n_ms) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (!latents || !frames) return fail(h, VD_ERR_INVALID_ARG, "latents/frames must not be NULL");
+    if (batch < 1 || batch > h->cfg.max_batch) return fail(h, VD_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
+    const size_t al = h->cfg.dtype == VD_BF16 ? 2 : 4;
+    if (((uintptr_t)latents % al) || ((uintptr_t)frames % al)) return fail(h, VD_ERR_INVALID_ARG, "latents/frames are misaligned for their dtype");
+    cudaStream_t s = (cudaStream_t)stream;
+    const int n = h->stop_after >= 0 ? std::min((int)h->steps.size(), h->stop_after + 1) : (int)h->steps.size();
+    std::vector<cudaEvent_t> ev;
+    if (ms) {
+        if (n_ms < (int)h->steps.size()) return fail(h, VD_ERR_INVALID_ARG, "ms array shorter than the number of steps");
+        ev.resize(n + 1);
+        for (auto& e : ev) {
+            cudaError_t ce = cudaEventCreate(&e);
+            if (ce != cudaSuccess) return cuda_fail(h, ce, "cudaEventCreate");
+        }
+        cudaEventRecord(ev[0], s);
+    }
+    for (int i = 0; i < n; ++i) {
+        cudaError_t e = launch_step(h, h->steps[i], batch, latents, v_prev, lambda, z_out, v_out, frames, s);
+        if (e != cudaSuccess) {
+            for (auto& x : ev) cudaEventDestroy(x);
+            return cuda_fail(h, e, h->steps[i].info.name);
+        }
+        if (ms) cudaEventRecord(ev[i + 1], s);
+    }
+    if (ms) {
+        cudaError_t e = cudaStreamSynchronize(s);
+        for (int i = 0; i < (int)h->steps.size(); ++i) ms[i] = 0.f;
+        if (e == cudaSuccess)
+            for (int i = 0; i < n; ++i) cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1]);
+        for (auto& x : ev) cudaEventDestroy(x);
+        if (e != cudaSuccess) return cuda_fail(h, e, "vd_profile synchronise");
+    }
+    return VD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+vd_status vd_query_workspace(const vd_config* cfg, size_t* bytes) {
+    std::string err;
+    vd_status st = validate_cfg(cfg, err);
+    if (st != VD_OK) return fail(nullptr, st, err);
+    if (!bytes) return fail(nullptr, VD_ERR_INVALID_ARG, "bytes is NULL");
+    vd_handle_s tmp;
+    tmp.cfg = *cfg;
+    Planner p(&tmp, nullptr);
+    p.plan();
+    *bytes = tmp.total;
+    return VD_OK;
+}
+
+vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_weights, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream, vd_handle* out) {
+    if (out) *out = nullptr;
+    std::string err;
+    vd_status st = validate_cfg(cfg, err);
+    if (st != VD_OK) return fail(nullptr, st, err);
+    if (!out) return fail(nullptr, VD_ERR_INVALID_ARG, "out is NULL");
+    if (!weights || n_weights <= 0) return fail(nullptr, VD_ERR_INVALID_ARG, "weights list is empty");
+    if (!workspace || ((uintptr_t)workspace % 256)) return fail(nullptr, VD_ERR_INVALID_ARG, "workspace must be non-NULL and 256-byte aligned");
+
+    int dev = 0, major = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "device query");
+    if (major != 10) return fail(nullptr, VD_ERR_UNSUPPORTED, "this library runs on sm_100 devices only");
+
+    vd_handle_s* h = new vd_handle_s();
+    h->cfg = *cfg;
+    h->ws = (char*)workspace;
+    h->ws_bytes = workspace_bytes;
+    Planner p(h, h->ws);
+    p.plan();
+    if (workspace_bytes < h->total) {
+        char msg[128];
+        snprintf(msg, sizeof(msg), "workspace too small: %zu bytes given, %zu needed", workspace_bytes, h->total);
+        delete h;
+        return fail(nullptr, VD_ERR_WORKSPACE, msg);
+    }
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    e = cudaMemsetAsync(h->ws + h->status_off, 0, 256, s);
+    if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "status memset"); }
+    for (const WeightJob& j : h->jobs) {
+        const vd_tensor* t = find_tensor(weights, n_weights, j.name);
+        if (!t) { std::string m = "missing weight tensor: " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
+        if (!t->dptr) { std::string m = "NULL pointer for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
+        if (t->dtype != cfg->dtype) { std::string m = "dtype of " + j.name + " differs from config.dtype"; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
+        int64_t want = j.kind == 0 ? (int64_t)j.Cout * j.Cin * j.taps : j.Cout;
+        int64_t have = 1;
+        if (t->ndim < 1 || t->ndim > 4) { std::string m = "bad ndim for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
+        for (int d = 0; d < t->ndim; ++d) have *= t->shape[d];
+        bool ok = have == want && t->shape[0] == j.Cout;
+        if (ok && j.kind == 0) ok = t->ndim >= 2 && t->shape[1] == j.Cin;
+        if (!ok) { std::string m = "shape mismatch for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
+        if (j.kind == 1) {
+            e = launch_to_f32(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, s);
+        } else if (j.tc) {
+            e = launch_pack_weight_tc(t->dptr, t->dtype, h->ws + j.dst_off, j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, s);
+        } else {
+            e = launch_pack_weight_simt(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, s);
+        }
+        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, j.name.c_str()); }
+    }
+    for (Step& st : h->steps) {
+        if (st.kind == VD_STEP_CONV && st.use_tc) {
+            e = conv_tc_prepare(st.conv, &st.tc);
+            if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "weight tensor map"); }
+        }
+    }
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "vd_create synchronise"); }
+    *out = h;
+    return VD_OK;
+}
+
+vd_status vd_decode(vd_handle h, const void* latents, void* frames, int32_t batch, void* cuda_stream) {
+    return decode_impl(h, latents, nullptr, 0.f, nullptr, nullptr, frames, batch, cuda_stream, nullptr, 0);
+}
+
+vd_status vd_decode_extrapolated(vd_handle h, const void* z_prev, const void* v_prev, float lambda, void* z_out,
+                                 void* v_out, void* frames, int32_t batch, void* cuda_stream) {
+    if (h && !v_prev) return fail(h, VD_ERR_INVALID_ARG, "v_prev must not be NULL");
+    return decode_impl(h, z_prev, v_prev, lambda, z_out, v_out, frames, batch, cuda_stream, nullptr, 0);
+}
+
+vd_status vd_decode_host(vd_handle h, const void* latents_host, void* frames_host, int32_t batch, void* cuda_stream) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (!latents_host || !frames_host) return fail(h, VD_ERR_INVALID_ARG, "host buffers must not be NULL");
+    if (batch < 1 || batch > h->cfg.max_batch) return fail(h, VD_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t es = elt(h->cfg.dtype);
+    const size_t lat_bytes = (size_t)batch * h->cfg.latent_channels * h->cfg.latent_h * h->cfg.latent_w * es;
+    const size_t frm_bytes = (size_t)batch * h->cfg.out_channels * h->cfg.latent_h * h->cfg.latent_w * 64 * es;
+    void* dl = h->ws + h->lat_stage_off;
+    void* df = h->ws + h->frm_stage_off;
+    cudaError_t e = cudaMemcpyAsync(dl, latents_host, lat_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "latents host-to-device copy");
+    vd_status st = decode_impl(h, dl, nullptr, 0.f, nullptr, nullptr, df, batch, cuda_stream, nullptr, 0);
+    if (st != VD_OK) return st;
+    e = cudaMemcpyAsync(frames_host, df, frm_bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "frames device-to-host copy");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(h, e, "vd_decode_host synchronise");
+    return VD_OK;
+}
+
+vd_status vd_get_status(vd_handle h) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    unsigned int word[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpy(word, h->ws + h->status_off, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e, "status read");
+    if (word[0] != 0) {
+        char msg[160];
+        snprintf(msg, sizeof(msg), "a kernel gave up on a bounded wait (code 0x%x, block %u, detail 0x%x)", word[0], word[1], word[2]);
+        return fail(h, VD_ERR_DEVICE_TIMEOUT, msg);
+    }
+    return VD_OK;
+}
+
+const char* vd_last_error(vd_handle h) { return h ? h->err.c_str() : g_last_error.c_str(); }
+
+vd_status vd_destroy(vd_handle h) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    delete h;
+    return VD_OK;
+}
+
+vd_status vd_num_steps(vd_handle h, int32_t* n) {
+    if (!h || !n) return fail(h, VD_ERR_INVALID_ARG, "NULL argument");
+    *n = (int32_t)h->steps.size();
+    return VD_OK;
+}
+
+vd_status vd_get_step(vd_handle h, int32_t index, vd_step_info* info) {
+    if (!h || !info) return fail(h, VD_ERR_INVALID_ARG, "NULL argument");
+    if (index < 0 || index >= (int)h->steps.size()) return fail(h, VD_ERR_INVALID_ARG, "step index out of range");
+    *info = h->steps[index].info;
+    return VD_OK;
+}
+
+vd_status vd_profile(vd_handle h, const void* latents, void* frames, int32_t batch, void* cuda_stream, float* ms,
+                     int32_t n_steps) {
+    if (!ms) return fail(h, VD_ERR_INVALID_ARG, "ms is NULL");
+    return decode_impl(h, latents, nullptr, 0.f, nullptr, nullptr, frames, batch, cuda_stream, ms, n_steps);
+}
+
+vd_status vd_debug_stop_after(vd_handle h, int32_t index) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (index < -1 || index >= (int)h->steps.size()) return fail(h, VD_ERR_INVALID_ARG, "step index out of range");
+    h->stop_after = index;
+    return VD_OK;
+}
+
+// ------------------------------------------------------------------ operator-level entry points
+static vd_status check_conv_desc(const vd_conv_desc* d) {
+    if (!d || d->struct_size != sizeof(vd_conv_desc)) return fail(nullptr, VD_ERR_INVALID_ARG, "bad conv descriptor");
+    if (d->batch < 0 || d->in_h < 1 || d->in_w < 1 || d->c_in < 1 || d->c_out < 1) return fail(nullptr, VD_ERR_INVALID_ARG, "bad conv sizes");
+    if (d->ksize != 1 && d->ksize != 3) return fail(nullptr, VD_ERR_INVALID_ARG, "ksize must be 1 or 3");
+    if ((d->in_dtype != VD_F32 && d->in_dtype != VD_BF16) || (d->out_dtype != VD_F32 && d->out_dtype != VD_BF16))
+        return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
+    if (d->impl < VD_IMPL_AUTO || d->impl > VD_IMPL_TC) return fail(nullptr, VD_ERR_INVALID_ARG, "bad impl");
+    return VD_OK;
+}
+
+static ConvArgs conv_args_from_desc(const vd_conv_desc* d) {
+    ConvArgs a{};
+    a.B = d->batch; a.Hs = d->in_h; a.Ws = d->in_w;
+    a.H = d->upsample ? 2 * d->in_h : d->in_h;
+    a.W = d->upsample ? 2 * d->in_w : d->in_w;
+    a.Cin = d->c_in; a.Cout = d->c_out; a.ksize = d->ksize; a.upsample = d->upsample ? 1 : 0; a.silu = d->silu ? 1 : 0;
+    a.in_dtype = d->in_dtype; a.out_dtype = d->out_dtype; a.out_nchw = d->out_nchw ? 1 : 0;
+    a.bf16_operands = d->bf16_operands ? 1 : 0;
+    return a;
+}
+
+static vd_status resolve_impl(const vd_conv_desc* d, const ConvArgs& a, bool* tc) {
+    ConvArgs probe = a;
+    probe.B = 1;
+    const bool can = a.bf16_operands && conv_tc_supported(probe);
+    if (d->impl == VD_IMPL_TC && !can) return fail(nullptr, VD_ERR_UNSUPPORTED, "the tensor-core convolution does not support this shape");
+    *tc = d->impl == VD_IMPL_TC || (d->impl == VD_IMPL_AUTO && can);
+    return VD_OK;
+}
+
+vd_status vd_conv_packed_weight_bytes(const vd_conv_desc* d, size_t* bytes) {
+    vd_status st = check_conv_desc(d);
+    if (st != VD_OK) return st;
+    if (!bytes) return fail(nullptr, VD_ERR_INVALID_ARG, "bytes is NULL");
+    bool tc;
+    st = resolve_impl(d, conv_args_from_desc(d), &tc);
+    if (st != VD_OK) return st;
+    const int taps = d->ksize * d->ksize;
+    *bytes = tc ? conv_tc_packed_bytes(d->c_out, d->c_in, taps) : (size_t)taps * d->c_in * d->c_out * 4;
+    return VD_OK;
+}
+
+vd_status vd_conv_pack_weight(const vd_conv_desc* d, const void* w_oihw, int32_t w_dtype, void* packed, void* cuda_stream) {
+    vd_status st = check_conv_desc(d);
+    if (st != VD_OK) return st;
+    if (!w_oihw || !packed) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
+    if (w_dtype != VD_F32 && w_dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
+    bool tc;
+    st = resolve_impl(d, conv_args_from_desc(d), &tc);
+    if (st != VD_OK) return st;
+    const int taps = d->ksize * d->ksize;
+    cudaError_t e = tc ? launch_pack_weight_tc(w_oihw, w_dtype, packed, d->c_out, d->c_in, taps, d->c_out, 0, (cudaStream_t)cuda_stream)
+                       : launch_pack_weight_simt(w_oihw, w_dtype, (float*)packed, d->c_out, d->c_in, taps, d->c_out, 0, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_conv_pack_weight");
+}
+
+vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* w_packed, const float* bias, const float* scale,
+                       const float* shift, const float* residual, void* y, void* cuda_stream) {
+    vd_status st = check_conv_desc(d);
+    if (st != VD_OK) return st;
+    if (!x || !w_packed || !y) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
+    if ((scale == nullptr) != (shift == nullptr)) return fail(nullptr, VD_ERR_INVALID_ARG, "scale and shift go together");
+    if (d->batch == 0) return VD_OK;
+    ConvArgs a = conv_args_from_desc(d);
+    a.x = x; a.w = w_packed; a.bias = bias; a.scale = scale; a.shift = shift; a.residual = residual; a.y = y;
+    bool tc;
+    st = resolve_impl(d, a, &tc);
+    if (st != VD_OK) return st;
+    cudaError_t e;
+    if (tc) {
+        ConvTcPlan plan{};
+        e = conv_tc_prepare(a, &plan);
+        if (e == cudaSuccess) e = launch_conv_tc(a, plan, nullptr, (cudaStream_t)cuda_stream);
+    } else {
+        e = launch_conv_simt(a, (cudaStream_t)cuda_stream);
+    }
+    return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_conv2d");
+}
+
+size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups) {
+    if (batch < 1 || groups < 1) return 0;
+    return (size_t)batch * kGnMaxChunks * groups * 4 * sizeof(float);
+}
+
+vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w, int32_t c, int32_t groups,
+                         float eps, const float* gamma, const float* beta, float* scale, float* shift, void* scratch,
+                         void* cuda_stream) {
+    if (!x || !gamma || !beta || !scale || !shift || !scratch) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
+    if (dtype != VD_F32 && dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
+    if (batch < 0 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups != 0 || (c / groups) % 4 != 0 || c > 1024)
+        return fail(nullptr, VD_ERR_INVALID_ARG, "bad GroupNorm sizes (groups must hold a multiple of 4 channels)");
+    if (batch == 0) return VD_OK;
+    GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch};
+    cudaError_t e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_gn_stats");
+}
+
+vd_status vd_op_attention(const void* q, const void* k, const void* v, void* o, int32_t dtype, int32_t batch,
+                          int32_t tokens, int32_t channels, int32_t ld_qkv, int32_t ld_o, float scale, int32_t impl,
+                          void* cuda_stream) {
+    if (!q || !k || !v || !o) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
+    if (dtype != VD_F32 && dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
+    if (batch < 0 || tokens < 1 || channels < 32 || channels % 32 != 0 || channels > 512 || ld_qkv < channels || ld_o < channels)
+        return fail(nullptr, VD_ERR_INVALID_ARG, "bad attention sizes");
+    if (impl < VD_IMPL_AUTO || impl > VD_IMPL_TC) return fail(nullptr, VD_ERR_INVALID_ARG, "bad impl");
+    if (batch == 0) return VD_OK;
+    AttnArgs a{q, k, v, o, dtype, batch, tokens, channels, ld_qkv, ld_o, scale};
+    const bool can = attn_tc_supported(a);
+    if (impl == VD_IMPL_TC && !can) return fail(nullptr, VD_ERR_UNSUPPORTED, "the tensor-core attention does not support this shape");
+    const bool tc = impl == VD_IMPL_TC || (impl == VD_IMPL_AUTO && can);
+    cudaError_t e = tc ? launch_attn_tc(a, nullptr, (cudaStream_t)cuda_stream) : launch_attn_simt(a, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_attention");
+}
+
+}  // extern "C"

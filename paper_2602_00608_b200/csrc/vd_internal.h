@@ -1,0 +1,85 @@
+// Internal declarations shared by the translation units of libvd.so (not part of the ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vd.h"
+
+namespace vd {
+
+// One fused convolution launch: y = conv(pad0(up2x?(act(x*scale+shift)))) + bias (+ residual).
+struct ConvArgs {
+    const void* x;          // NHWC [B,Hs,Ws,Cin], in_dtype
+    const void* w;          // packed weights (layout depends on the implementation)
+    const float* bias;      // [Cout] or null
+    const float* scale;     // [B,Cin] or null
+    const float* shift;     // [B,Cin] or null
+    const float* residual;  // fp32 NHWC [B,H,W,Cout] or null
+    void* y;                // out_dtype, NHWC [B,H,W,Cout] or NCHW [B,Cout,H,W]
+    int B, Hs, Ws;          // source resolution
+    int H, W;               // output resolution (= source, or 2x source with upsample)
+    int Cin, Cout, ksize, upsample, silu;
+    int in_dtype, out_dtype, out_nchw, bf16_operands;
+};
+
+struct GnArgs {
+    const void* x;          // NHWC [B,H,W,C]
+    int dtype;
+    int B, P, C, G;         // P = H*W
+    float eps;
+    const float* gamma;     // [C]
+    const float* beta;      // [C]
+    float* scale;           // [B,C]
+    float* shift;           // [B,C]
+    float* partial;         // [B, kGnMaxChunks, G, 4] scratch
+};
+constexpr int kGnMaxChunks = 1024;
+
+struct AttnArgs {
+    const void* q; const void* k; const void* v; void* o;
+    int dtype;
+    int B, T, C, ld_qkv, ld_o;
+    float scale;
+};
+
+struct IngestArgs {
+    const void* z;          // NCHW latents (or z_prev when v_prev is set)
+    const void* v_prev;     // null, or the motion vector for z = z_prev + lambda*v_prev
+    void* z_out;            // optional NCHW copy of the extrapolated latents
+    void* v_out;            // optional NCHW new motion vector z - z_prev
+    float lambda;
+    float* x;               // fp32 NHWC [B,h,w,C]
+    int dtype, B, C, h, w;
+};
+
+// ---- FFMA kernels (kernels_simt.cu)
+cudaError_t launch_ingest(const IngestArgs& a, cudaStream_t s);
+cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s);          // two launches
+cudaError_t launch_conv_simt(const ConvArgs& a, cudaStream_t s);
+cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
+// OIHW (or [out,in]) weight of dtype `w_dtype` -> fp32 [tap][Cin][Cout]
+// (Cout rows are written at column offset cout_offset of a packed matrix cout_total wide)
+cudaError_t launch_pack_weight_simt(const void* w, int w_dtype, float* packed, int Cout, int Cin, int taps,
+                                    int cout_total, int cout_offset, cudaStream_t s);
+// any vector of dtype -> fp32
+cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cudaStream_t s);
+
+// ---- tcgen05 kernels (conv_tc.cu, attn_tc.cu)
+bool conv_tc_supported(const ConvArgs& a);
+size_t conv_tc_packed_bytes(int Cout, int Cin, int taps);
+// OIHW weight (bf16) -> bf16 [tap][Cout_pad][Cin] (K-major rows for the B operand)
+cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int Cout, int Cin, int taps,
+                                  int cout_total, int cout_offset, cudaStream_t s);
+// Launch-invariant state of one tensor-core convolution: the TMA descriptor of its packed weights.
+struct alignas(64) ConvTcPlan {
+    unsigned char tmap[128];
+    int bn;
+    int valid;
+};
+cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
+cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
+bool attn_tc_supported(const AttnArgs& a);
+cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
+
+}  // namespace vd

@@ -1,0 +1,160 @@
+"""End-to-end parity of vd_decode against the oracle on the benchmark configurations, through
+the C ABI, on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+
+from tests.util import BF16_MAX_ABS, BF16_REL_L2, F32_REL_L2, max_abs, rel_l2
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from oracle import ref
+    from paper_2602_00608_b200 import binding, synth
+    return torch, ref, binding, synth
+
+
+def _decode(env, wl, z, flags=0, max_batch=None):
+    torch, ref, vd, synth = env
+    wts = synth.workload_weights(wl)
+    dec = vd.Decoder(wl.arch, wl.dtype, z.shape[2], z.shape[3], max_batch or z.shape[0], wl.groups, wl.eps, wts, flags)
+    zt = torch.from_numpy(z).to("cuda:0", dec.dtype)
+    got = dec.decode(zt)
+    torch.cuda.synchronize()
+    dec.check_status()
+    return dec, got, wts
+
+
+def test_config1_tiny_fp32(env):
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[1]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z)
+    want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+    assert got.shape == (1, 3, 64, 64) and got.dtype == torch.float32
+    assert rel_l2(got.cpu().numpy(), want) <= F32_REL_L2
+
+
+def test_tiny_fp32_odd_size_batch3(env):
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[1]
+    z = synth.workload_latents(wl, batch=3, h=5, w=7)
+    dec, got, wts = _decode(env, wl, z)
+    want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+    assert rel_l2(got.cpu().numpy(), want) <= F32_REL_L2
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_config2_sdvae_bf16_64x64(env, flags):
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[2]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z, flags)
+    want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+    g = got.float().cpu().numpy()
+    assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+
+
+def test_sdvae_fp32_path_matches_oracle(env):
+    # the fp32 FFMA path on the full-width layout (attention and shortcuts included)
+    torch, ref, vd, synth = env
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS[2], dtype="f32")
+    z = synth.workload_latents(wl, batch=2, h=5, w=6)
+    dec, got, wts = _decode(env, wl, z)
+    want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+    assert rel_l2(got.cpu().numpy(), want) <= F32_REL_L2
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_sdvae_bf16_ragged_tiles_batch2(env, flags):
+    # 20x28 latents: every level's width/height leaves a ragged last tile; two frames
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[3]
+    z = synth.workload_latents(wl, batch=2, h=20, w=28)
+    dec, got, wts = _decode(env, wl, z, flags)
+    want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+    g = got.float().cpu().numpy()
+    assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+    # batch independence and run-to-run determinism
+    again = dec.decode(torch.from_numpy(z).to("cuda:0", dec.dtype))
+    one = dec.decode(torch.from_numpy(z[1:2]).to("cuda:0", dec.dtype))
+    torch.cuda.synchronize()
+    assert torch.equal(again, got)
+    assert torch.equal(one[0], got[1])
+
+
+@pytest.mark.parametrize("idx", [3, 4, 5])
+def test_full_size_configs_against_sampled_oracle_frames(env, idx):
+    """Full-size workloads in the benchmark's launch configuration; the oracle frames were computed
+    ahead of time by tests/golden/make_golden.py (oracle only) and sampled at fixed pixels."""
+    torch, ref, vd, synth = env
+    path = os.path.join(GOLDEN, f"frames_cfg{idx}.npz")
+    if not os.path.exists(path):
+        pytest.skip(f"{path} not generated")
+    gold = np.load(path)
+    wl = synth.WORKLOADS[idx]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z)
+    pos = gold["positions"]
+    g = got.float().cpu().numpy()
+    assert g.shape == (wl.batch, 3, wl.out_h, wl.out_w)
+    sampled = g[:, :, pos[:, 0], pos[:, 1]]
+    for b in range(wl.batch):
+        r, m = rel_l2(sampled[b], gold["values"][b]), max_abs(sampled[b], gold["values"][b])
+        assert r <= BF16_REL_L2 and m <= BF16_MAX_ABS, (b, r, m)
+        # whole-frame statistics as a property check on the pixels that were not sampled
+        std = float(g[b].astype(np.float64).std())
+        assert abs(std - gold["stats"][b, 1]) <= 0.01 * gold["stats"][b, 1]
+    dec.check_status()
+
+
+def test_host_buffer_decode_and_extrapolation(env):
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[2]
+    z = synth.workload_latents(wl, batch=2)
+    dec, got, wts = _decode(env, wl, z)
+    zh = torch.from_numpy(z).to(dec.dtype).pin_memory()
+    fh = torch.empty((2, 3, 64, 64), dtype=dec.dtype).pin_memory()
+    dec.decode_host(zh, fh)
+    assert torch.equal(fh, got.cpu())
+    # Algorithm 2, hit branch: z = z_prev + lambda*v_prev decoded in one call
+    v = synth.round_to_bf16((0.1 * np.random.default_rng(1).standard_normal(z.shape)).astype(np.float32))
+    lam = 0.5
+    z_want, v_want = ref.extrapolate(z, v, lam)
+    frames, z_new, v_new = dec.decode_extrapolated(torch.from_numpy(z).to("cuda:0", dec.dtype),
+                                                   torch.from_numpy(v).to("cuda:0", dec.dtype), lam)
+    torch.cuda.synchronize()
+    assert max_abs(z_new.float().cpu().numpy(), z_want) <= 2 ** -8 * np.abs(z_want).max()
+    assert max_abs(v_new.float().cpu().numpy(), v_want) <= 2 ** -8 * np.abs(z_want).max()
+    want = ref.decode(wl.arch, wts, z_new.float().cpu().numpy(), wl.groups, wl.eps)
+    g = frames.float().cpu().numpy()
+    assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+
+
+def test_decode_argument_errors(env):
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[1]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z)
+    import ctypes
+    l = vd.lib()
+    assert l.vd_decode(dec.handle, None, ctypes.c_void_p(got.data_ptr()), 1, None) == vd.VD_ERR_INVALID_ARG
+    assert l.vd_decode(dec.handle, ctypes.c_void_p(got.data_ptr()), ctypes.c_void_p(got.data_ptr()), 2, None) == vd.VD_ERR_INVALID_ARG
+    assert b"batch" in l.vd_last_error(dec.handle)
+    # missing weight / wrong shape / small workspace
+    bad = dict(wts)
+    del bad["conv_out.bias"]
+    with pytest.raises(vd.VdError) as e:
+        vd.Decoder(wl.arch, wl.dtype, 8, 8, 1, wl.groups, wl.eps, bad)
+    assert e.value.status == vd.VD_ERR_INVALID_ARG and "conv_out.bias" in str(e.value)
+    bad = dict(wts)
+    bad["conv_in.weight"] = bad["conv_in.weight"][:, :3]
+    with pytest.raises(vd.VdError) as e:
+        vd.Decoder(wl.arch, wl.dtype, 8, 8, 1, wl.groups, wl.eps, bad)
+    assert e.value.status == vd.VD_ERR_INVALID_ARG
