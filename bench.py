@@ -156,6 +156,7 @@ def main():
     ap.add_argument("--impl", default="vd", choices=["vd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="force the FFMA cross-check kernels")
+    ap.add_argument("--per-step", default=None, help="write a per-step table (name, ms, TFLOP/s, GB/s) to this file")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "vd" else args.warmup
 
@@ -242,6 +243,17 @@ def main():
     for _ in range(prof_runs):
         for i, v in enumerate(dec.profile(z, frames)):
             acc[i] += v / prof_runs
+    if args.per_step and rank == 0:
+        with open(args.per_step, "w") as f:
+            f.write(f"# {wl.name}: per-step device time (CUDA events around each step, mean of {prof_runs} decodes)\n")
+            f.write("# name kind impl ms TFLOP/s GB/s(as stored) roofline_us(bf16 contract)\n")
+            tf, bw = peaks["bf16_tflops"] * 1e12, peaks["hbm_gbs"] * 1e9
+            for s, ms in zip(steps, acc):
+                fl = s["flops_per_frame"] * wl.batch
+                by = s["bytes_per_frame"] * wl.batch + s["weight_bytes"]
+                ru, _, _ = contract_roofline_us([s], peaks, wl.batch, 2)
+                f.write(f"{s['name']:22s} {s['kind']} {s['impl']} {ms:9.4f} {fl / (ms * 1e-3) / 1e12 if ms > 0 else 0:9.1f} "
+                        f"{by / (ms * 1e-3) / 1e9 if ms > 0 else 0:9.1f} {ru * wl.batch:9.2f}\n")
     by_kind = {}
     for s, ms in zip(steps, acc):
         key = ("conv_tc" if s["impl"] else "conv_ffma") if s["kind"] == 2 else {0: "ingest", 1: "gn_stats", 3: "attention"}[s["kind"]]

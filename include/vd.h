@@ -210,10 +210,13 @@ VD_API vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int
 
 /* o[t,:] = sum_u softmax_u(scale * q[t,:].k[u,:]) v[u,:] for each batch item; q, k, v, o are
  * device rows of `dtype` with `ld` elements between consecutive tokens (so q, k, v may be
- * slices of one [tokens, 3C] tensor); tokens >= 1, channels = 512 for the tensor-core kernel. */
+ * slices of one [tokens, 3C] tensor); tokens >= 1.  The tensor-core kernel needs bf16, 512
+ * channels, 16-byte aligned pointers, ld multiples of 8, and `scratch`: device memory of
+ * vd_attention_scratch_bytes bytes (it holds V transposed); the FFMA kernel ignores scratch. */
+VD_API size_t vd_attention_scratch_bytes(int32_t batch, int32_t tokens, int32_t channels);
 VD_API vd_status vd_op_attention(const void* q, const void* k, const void* v, void* o, int32_t dtype,
                                  int32_t batch, int32_t tokens, int32_t channels, int32_t ld_qkv, int32_t ld_o,
-                                 float scale, int32_t impl, void* cuda_stream);
+                                 float scale, int32_t impl, void* scratch, void* cuda_stream);
 
 #ifdef __cplusplus
 }

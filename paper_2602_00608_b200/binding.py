@@ -24,7 +24,7 @@ EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
     "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
-    "vd_op_attention",
+    "vd_op_attention", "vd_attention_scratch_bytes",
 ]
 
 
@@ -89,9 +89,11 @@ def lib():
         l.vd_gn_scratch_bytes.argtypes = [c_int32, c_int32]
         l.vd_gn_scratch_bytes.restype = c_size_t
         l.vd_op_gn_stats.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp, vp]
-        l.vd_op_attention.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, vp]
+        l.vd_op_attention.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, vp, vp]
+        l.vd_attention_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
+        l.vd_attention_scratch_bytes.restype = c_size_t
         for name in EXPORTED:
-            if name not in ("vd_last_error", "vd_gn_scratch_bytes"):
+            if name not in ("vd_last_error", "vd_gn_scratch_bytes", "vd_attention_scratch_bytes"):
                 getattr(l, name).restype = c_int32
         _lib = l
     return _lib
@@ -297,8 +299,10 @@ def op_attention(qkv, channels: int, scale: float, impl=VD_IMPL_AUTO):
     b, t, c3 = qkv.shape
     assert c3 == 3 * channels and qkv.is_contiguous()
     o = torch.empty((b, t, channels), dtype=qkv.dtype, device=qkv.device)
+    scratch = torch.empty(max(16, lib().vd_attention_scratch_bytes(b, t, channels)), dtype=torch.uint8, device=qkv.device)
     es = qkv.element_size()
     base = qkv.data_ptr()
     _check(lib().vd_op_attention(c_void_p(base), c_void_p(base + channels * es), c_void_p(base + 2 * channels * es),
-                                 c_void_p(o.data_ptr()), _dt(qkv), b, t, channels, c3, channels, scale, impl, _stream_ptr()))
+                                 c_void_p(o.data_ptr()), _dt(qkv), b, t, channels, c3, channels, scale, impl,
+                                 c_void_p(scratch.data_ptr()), _stream_ptr()))
     return o

@@ -179,7 +179,7 @@ class Planner {
         s.kind = VD_STEP_ATTENTION;
         const int es = elt(act_dtype());
         s.attn = AttnArgs{ptr<void>(qkv_), ptr<void>(qkv_ + (size_t)C * es), ptr<void>(qkv_ + (size_t)2 * C * es),
-                          ptr<void>(attno_), act_dtype(), 0, H * W, C, 3 * C, C, 1.0f / sqrtf((float)C)};
+                          ptr<void>(attno_), act_dtype(), 0, H * W, C, 3 * C, C, 1.0f / sqrtf((float)C), ptr<void>(vt_)};
         s.use_tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && attn_tc_supported(s.attn);
         fill_info(s, p + ".core", s.use_tc, C, C, 0, 0, H, W, C, act_dtype(), 0, (long)attno_);
         const double T = (double)H * W;
@@ -241,6 +241,7 @@ class Planner {
         sbuf_ = max_s ? alloc((size_t)B * max_s * 4) : 0;
         qkv_ = qkv ? alloc((size_t)B * qkv * ae) : 0;
         attno_ = ao ? alloc((size_t)B * ao * ae) : 0;
+        vt_ = ao ? alloc(attn_tc_scratch_bytes(B, (int)P0, 512)) : 0;
         h_->lat_stage_off = alloc((size_t)B * P0 * lc * elt(cfg_.dtype));
         h_->frm_stage_off = alloc((size_t)B * P0 * 64 * cfg_.out_channels * elt(cfg_.dtype));
 
@@ -306,7 +307,7 @@ class Planner {
     char* base_;
     const vd_config& cfg_;
     size_t cur_ = 0;
-    size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, sbuf_ = 0, qkv_ = 0, attno_ = 0;
+    size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, sbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
     int cur_x_ = 0;
 };
@@ -668,17 +669,22 @@ vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h,
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_gn_stats");
 }
 
+size_t vd_attention_scratch_bytes(int32_t batch, int32_t tokens, int32_t channels) {
+    if (batch < 1 || tokens < 1 || channels < 1) return 0;
+    return attn_tc_scratch_bytes(batch, tokens, channels);
+}
+
 vd_status vd_op_attention(const void* q, const void* k, const void* v, void* o, int32_t dtype, int32_t batch,
                           int32_t tokens, int32_t channels, int32_t ld_qkv, int32_t ld_o, float scale, int32_t impl,
-                          void* cuda_stream) {
+                          void* scratch, void* cuda_stream) {
     if (!q || !k || !v || !o) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
     if (dtype != VD_F32 && dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
     if (batch < 0 || tokens < 1 || channels < 32 || channels % 32 != 0 || channels > 512 || ld_qkv < channels || ld_o < channels)
         return fail(nullptr, VD_ERR_INVALID_ARG, "bad attention sizes");
     if (impl < VD_IMPL_AUTO || impl > VD_IMPL_TC) return fail(nullptr, VD_ERR_INVALID_ARG, "bad impl");
     if (batch == 0) return VD_OK;
-    AttnArgs a{q, k, v, o, dtype, batch, tokens, channels, ld_qkv, ld_o, scale};
-    const bool can = attn_tc_supported(a);
+    AttnArgs a{q, k, v, o, dtype, batch, tokens, channels, ld_qkv, ld_o, scale, scratch};
+    const bool can = attn_tc_supported(a) && scratch != nullptr;
     if (impl == VD_IMPL_TC && !can) return fail(nullptr, VD_ERR_UNSUPPORTED, "the tensor-core attention does not support this shape");
     const bool tc = impl == VD_IMPL_TC || (impl == VD_IMPL_AUTO && can);
     cudaError_t e = tc ? launch_attn_tc(a, nullptr, (cudaStream_t)cuda_stream) : launch_attn_simt(a, (cudaStream_t)cuda_stream);

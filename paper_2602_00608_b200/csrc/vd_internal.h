@@ -41,6 +41,7 @@ struct AttnArgs {
     int dtype;
     int B, T, C, ld_qkv, ld_o;
     float scale;
+    void* vt;               // scratch for the tensor-core kernel: V transposed, [B][C][round_up(T,64)] bf16
 };
 
 struct IngestArgs {
@@ -80,6 +81,7 @@ struct alignas(64) ConvTcPlan {
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
 bool attn_tc_supported(const AttnArgs& a);
+size_t attn_tc_scratch_bytes(int B, int T, int C);
 cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
 
 }  // namespace vd

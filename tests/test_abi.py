@@ -88,7 +88,7 @@ def test_null_arguments_are_rejected_without_a_device(vd):
     assert l.vd_num_steps(None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_op_conv2d(None, None, None, None, None, None, None, None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_op_gn_stats(None, 0, 1, 1, 1, 4, 1, 1e-6, None, None, None, None, None, None) == vd.VD_ERR_INVALID_ARG
-    assert l.vd_op_attention(None, None, None, None, 0, 1, 1, 32, 32, 32, 1.0, 0, None) == vd.VD_ERR_INVALID_ARG
+    assert l.vd_op_attention(None, None, None, None, 0, 1, 1, 32, 32, 32, 1.0, 0, None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_gn_scratch_bytes(0, 32) == 0
     assert b"NULL" in l.vd_last_error(None) or l.vd_last_error(None)
 

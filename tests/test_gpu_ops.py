@@ -220,3 +220,38 @@ def test_conv_tc_real_layer_shape_sampled(env):
         a0, a1, b0, b1 = max(i0 - 1, 0), min(i0 + 9, H), max(j0 - 1, 0), min(j0 + 9, W)
         want = ref.conv2d(x[:, :, a0:a1, b0:b1], w, bias)[:, :, i0 - a0:i0 - a0 + 8, j0 - b0:j0 - b0 + 8]
         assert rel_l2(got[:, :, i0:i0 + 8, j0:j0 + 8], want) <= 1e-4, (i0, j0)
+
+
+# ------------------------------------------------------------------ tensor-core attention
+@pytest.mark.parametrize("B,T", [(1, 64), (1, 128), (2, 300), (1, 1000), (1, 129)])
+def test_attention_tc_matches_oracle(env, B, T):
+    _, _, vd, _ = env
+    got, want = _attn_case(env, 51, B, T, 512, True, vd.VD_IMPL_TC)
+    # bf16 probabilities and bf16 output: two roundings of 2^-9 relative
+    assert rel_l2(got, want) <= 6e-3
+    got2, _ = _attn_case(env, 51, B, T, 512, True, vd.VD_IMPL_SIMT)
+    assert rel_l2(got, got2) <= 6e-3
+
+
+def test_attention_tc_growing_scores_trigger_rescaling(env):
+    """Keys ordered so that the row maximum keeps growing by more than the rescaling threshold from
+    one key tile to the next: exercises the accumulator rescale path against the oracle."""
+    torch, ref, vd, synth = env
+    T, C = 640, 512
+    r = _rng(52)
+    q = r.standard_normal((1, T, C)).astype(np.float32)
+    k = r.standard_normal((1, T, C)).astype(np.float32) * 0.05
+    ramp = (np.arange(T) // 128).astype(np.float32)[None, :, None]         # + one step per key tile
+    k = k + ramp * 0.6 * np.sign(q.mean(axis=1, keepdims=True))             # scores grow with the tile index
+    q = q + 0.5 * np.sign(q.mean(axis=1, keepdims=True))
+    v = r.standard_normal((1, T, C)).astype(np.float32)
+    qkv = synth.round_to_bf16(np.concatenate([q, k, v], axis=2))
+    scale = 1.0 / math.sqrt(C)
+    qq, kk, vv = (np.ascontiguousarray(qkv[:, :, i * C:(i + 1) * C].transpose(0, 2, 1)) for i in range(3))
+    want, probs = ref.attention_core(qq, kk, vv, scale, return_probs=True)
+    s = np.einsum("ct,cu->tu", qq[0].astype(np.float64), kk[0].astype(np.float64)) * scale
+    tile_max = np.stack([s[:, i:i + 128].max(axis=1) for i in range(0, T, 128)], axis=1)
+    assert np.median(np.diff(tile_max, axis=1)) * 1.4427 > 8.0              # really beyond the threshold
+    got = vd.op_attention(torch.from_numpy(qkv).cuda().bfloat16(), C, scale, vd.VD_IMPL_TC)
+    torch.cuda.synchronize()
+    assert rel_l2(got.float().cpu().numpy(), want.transpose(0, 2, 1)) <= 6e-3
