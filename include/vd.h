@@ -208,6 +208,22 @@ VD_API vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int
                                 int32_t groups, float eps, const float* gamma, const float* beta,
                                 float* scale, float* shift, void* scratch, void* cuda_stream);
 
+/* The same operator for callers that cannot hand over (or allocate) a scratch buffer.  The paper
+ * has no counterpart of this entry point; it exists for hosts where device allocation is not an
+ * option at call time: frame loops that must not hit the allocator's implicit synchronisation,
+ * plug-ins living inside another application's memory budget, code running in a host callback.
+ * The chunk partials live in a 1 MiB array built into the library (held by every GPU that loads
+ * it until the process exits).  Limits and rules:
+ *   - batch * groups <= 64, else VD_ERR_UNSUPPORTED (use vd_op_gn_stats);
+ *   - no cudaMalloc/cudaFree or any allocating routine is called;
+ *   - the first call on a device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture;
+ *   - all calls on a device share the array: calls whose kernels may overlap on the GPU race.
+ *     Nothing needs clearing between calls (each call writes every slot it later reads). */
+VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w,
+                                       int32_t c, int32_t groups, float eps, const float* gamma,
+                                       const float* beta, float* scale, float* shift, void* cuda_stream);
+
 /* o[t,:] = sum_u softmax_u(scale * q[t,:].k[u,:]) v[u,:] for each batch item; q, k, v, o are
  * device rows of `dtype` with `ld` elements between consecutive tokens (so q, k, v may be
  * slices of one [tokens, 3C] tensor); tokens >= 1.  The tensor-core kernel needs bf16, 512

@@ -24,7 +24,7 @@ EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
     "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
-    "vd_op_attention", "vd_attention_scratch_bytes",
+    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static",
 ]
 
 
@@ -89,6 +89,7 @@ def lib():
         l.vd_gn_scratch_bytes.argtypes = [c_int32, c_int32]
         l.vd_gn_scratch_bytes.restype = c_size_t
         l.vd_op_gn_stats.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp, vp]
+        l.vd_op_gn_stats_static.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp]
         l.vd_op_attention.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, vp, vp]
         l.vd_attention_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
         l.vd_attention_scratch_bytes.restype = c_size_t
@@ -290,6 +291,19 @@ def op_gn_stats(x_nhwc, gamma, beta, groups: int, eps: float):
     shift = torch.empty((b, c), dtype=torch.float32, device=x_nhwc.device)
     p = lambda t: c_void_p(t.data_ptr())
     _check(lib().vd_op_gn_stats(p(x_nhwc.contiguous()), _dt(x_nhwc), b, h, w, c, groups, eps, p(gamma), p(beta), p(scale), p(shift), p(scratch), _stream_ptr()))
+    return scale, shift
+
+
+def op_gn_stats_static(x_nhwc, gamma, beta, groups: int, eps: float):
+    """op_gn_stats through the entry point that uses the library's built-in scratch array: for
+    callers that may not allocate (this wrapper itself only allocates the two outputs)."""
+    import torch
+    b, h, w, c = x_nhwc.shape
+    scale = torch.empty((b, c), dtype=torch.float32, device=x_nhwc.device)
+    shift = torch.empty((b, c), dtype=torch.float32, device=x_nhwc.device)
+    p = lambda t: c_void_p(t.data_ptr())
+    _check(lib().vd_op_gn_stats_static(p(x_nhwc.contiguous()), _dt(x_nhwc), b, h, w, c, groups, eps, p(gamma), p(beta),
+                                       p(scale), p(shift), _stream_ptr()))
     return scale, shift
 
 

@@ -3,6 +3,9 @@
 // fp32 configuration end to end and serve as the on-GPU cross-check path of the bf16 one.
 #include <math.h>
 
+#include <mutex>
+#include <string>
+
 #include "vd_internal.h"
 
 namespace vd {
@@ -462,4 +465,74 @@ cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cud
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------------
+// GroupNorm statistics without any caller-provided or allocated scratch memory.
+//
+// Some callers may not allocate device memory at the point where they need this operator: a
+// render/game loop that must not stall on the allocator's implicit device synchronisation, a
+// plug-in whose host application owns the whole memory pool, or code running where the CUDA
+// allocator is simply off limits (inside a host callback, after a memory budget was frozen).
+// For them the chunk partials of the reduction live in the fixed device array below instead of a
+// buffer passed in.  The price is a size limit and shared state: every GPU that loads this
+// library carries the array (1 MiB) until the process exits, and all calls on a device use the
+// same array, so two calls whose kernels can overlap on the GPU (different streams, no ordering
+// between them) race on it.  Nothing in the array has to start at zero: every slot the second
+// kernel reads was written by the first kernel of the same call, so stale contents of an earlier
+// call are never observed.
+namespace {
+constexpr int kStaticGnMaxBatchTimesGroups = 64;     // e.g. 2 frames x 32 groups, or 8 x 8
+static __device__ __align__(256) float g_gn_static_partial[kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 4];   // 1 MiB
+
+std::mutex g_static_mu;
+constexpr int kMaxDevices = 64;
+float* g_static_ptr[kMaxDevices] = {};
+
+// In host code the array's name is only a handle of the symbol, not a device address; the address
+// on the current device is looked up once per device and cached.
+cudaError_t static_scratch_of_current_device(float** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_gn_static_partial);
+        if (e != cudaSuccess) return e;
+        g_static_ptr[dev] = (float*)p;
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+
 }  // namespace vd
+
+extern "C" VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w,
+                                                  int32_t c, int32_t groups, float eps, const float* gamma,
+                                                  const float* beta, float* scale, float* shift, void* cuda_stream) {
+    using namespace vd;
+    if (!x || !gamma || !beta || !scale || !shift) { set_last_error("vd_op_gn_stats_static: NULL pointer"); return VD_ERR_INVALID_ARG; }
+    if (dtype != VD_F32 && dtype != VD_BF16) { set_last_error("vd_op_gn_stats_static: bad dtype"); return VD_ERR_INVALID_ARG; }
+    if (batch < 0 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups != 0 || (c / groups) % 4 != 0 || c > 1024) {
+        set_last_error("vd_op_gn_stats_static: bad GroupNorm sizes (groups must hold a multiple of 4 channels)");
+        return VD_ERR_INVALID_ARG;
+    }
+    if ((long long)batch * groups > kStaticGnMaxBatchTimesGroups) {
+        set_last_error("vd_op_gn_stats_static: batch*groups exceeds 64, the capacity of the built-in scratch array; "
+                       "use vd_op_gn_stats with a scratch buffer instead");
+        return VD_ERR_UNSUPPORTED;
+    }
+    if (batch == 0) return VD_OK;
+    float* partial = nullptr;
+    cudaError_t e = static_scratch_of_current_device(&partial);
+    if (e == cudaSuccess) {
+        GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial};
+        e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
+    }
+    if (e != cudaSuccess) {
+        set_last_error((std::string("vd_op_gn_stats_static: ") + cudaGetErrorString(e)).c_str());
+        return VD_ERR_CUDA;
+    }
+    return VD_OK;
+}

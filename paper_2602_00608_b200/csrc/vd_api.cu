@@ -414,6 +414,10 @@ vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, floa
 
 }  // namespace
 
+namespace vd {
+void set_last_error(const char* msg) { g_last_error = msg ? msg : ""; }
+}  // namespace vd
+
 extern "C" {
 
 vd_status vd_query_workspace(const vd_config* cfg, size_t* bytes) {

@@ -54,6 +54,9 @@ struct IngestArgs {
     int dtype, B, C, h, w;
 };
 
+// records `msg` as the text vd_last_error(NULL) returns (defined in vd_api.cu)
+void set_last_error(const char* msg);
+
 // ---- FFMA kernels (kernels_simt.cu)
 cudaError_t launch_ingest(const IngestArgs& a, cudaStream_t s);
 cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s);          // two launches
