@@ -59,11 +59,23 @@ def contract_roofline_us(steps, peaks, batch, stream_bytes=2):
             elif s["kind"] == 2:
                 src = P // 4 if s["upsample"] else P
                 by = src * s["c_in"] * stream_bytes + P * s["c_out"] * stream_bytes
-                if s["name"].endswith(".conv2") or s["name"].endswith(".o"):
+                if s["has_residual"] or s.get("c_in2", 0) > 0:
                     by += P * s["c_out"] * stream_bytes
             else:
                 by = 4 * P * s["c_in"] * stream_bytes
-        by += s["weight_bytes"] / batch
+        wb = s["weight_bytes"]
+        if s.get("c_in2", 0) > 0 and stream_bytes is not None:
+            # a fused 1x1 shortcut: the contract counts it as a layer of its own (in, out, weights once)
+            P = s["out_h"] * s["out_w"]
+            fl2 = 2.0 * s["c_in2"] * s["c_out"] * P
+            wb2 = s["c_in2"] * s["c_out"] * 2
+            by2 = P * s["c_in2"] * stream_bytes + P * s["c_out"] * stream_bytes + wb2 / batch
+            total += max(fl2 / tf, by2 / bw)
+            flops += fl2
+            byts += by2
+            fl -= fl2
+            wb -= wb2
+        by += wb / batch
         total += max(fl / tf, by / bw)
         flops += fl
         byts += by

@@ -149,6 +149,8 @@ typedef struct {
     double flops_per_frame;     /* 2*taps*Cin*Cout*P for a conv, 4*T*T*C for attention, 0 otherwise */
     double bytes_per_frame;     /* algorithmic HBM bytes as stored (inputs once, output once, residual once) */
     double weight_bytes;        /* parameter bytes read once per launch (shared by the batch) */
+    int32_t c_in2;              /* > 0: a 1x1 shortcut on a second input of c_in2 channels is fused in */
+    int32_t has_residual;       /* 1: an fp32 residual tensor is added in the epilogue */
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);

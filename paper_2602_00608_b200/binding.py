@@ -43,7 +43,8 @@ class VdStepInfo(Structure):
                 ("c_in", c_int32), ("c_out", c_int32), ("ksize", c_int32), ("upsample", c_int32),
                 ("out_h", c_int32), ("out_w", c_int32), ("out_channels", c_int32), ("out_dtype", c_int32),
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
-                ("bytes_per_frame", c_double), ("weight_bytes", c_double)]
+                ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
+                ("has_residual", c_int32)]
 
 
 class VdConvDesc(Structure):

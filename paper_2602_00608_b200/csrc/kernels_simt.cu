@@ -162,37 +162,45 @@ __global__ void __launch_bounds__(kGnThreads) gn_partial_kernel(GnArgs a, int ch
     }
 }
 
-// Pass B: one warp per (sample, group) merges the chunk partials (lanes stride over the chunks,
-// then a shuffle tree), and folds the statistics with the affine parameters into per-(sample,
-// channel) scale and shift.
-__global__ void gn_finalize_kernel(GnArgs a, int chunks) {
-    const int n = blockIdx.x;
+// Pass B: one block per (group, sample) merges that group's chunk partials (independent loads
+// first, then a fixed-order tree), and folds the statistics with the affine parameters into
+// per-(sample, channel) scale and shift.
+constexpr int kGnFinalThreads = 128;
+__global__ void __launch_bounds__(kGnFinalThreads) gn_finalize_kernel(GnArgs a, int chunks) {
+    __shared__ Moments sm[kGnFinalThreads / 32];
+    const int g = blockIdx.x, n = blockIdx.y;
     const int cpg = a.C / a.G;
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32, nwarps = blockDim.x / 32;
-    for (int g = warp; g < a.G; g += nwarps) {
-        Moments m = {0.f, 0.f, 0.f};
-        for (int k = lane; k < chunks; k += 32) {
-            const float4 p = *(const float4*)(a.partial + (((size_t)n * kGnMaxChunks + k) * a.G + g) * 4);
-            m = merge(m, Moments{p.x, p.y, p.z});
-        }
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    constexpr int PER = kGnMaxChunks / kGnFinalThreads;          // 8 partials per thread at most
+    float4 p[PER];
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            Moments o;
-            o.n = __shfl_xor_sync(0xffffffffu, m.n, d);
-            o.mean = __shfl_xor_sync(0xffffffffu, m.mean, d);
-            o.m2 = __shfl_xor_sync(0xffffffffu, m.m2, d);
-            m = merge(m, o);
-        }
-        const float cnt = __shfl_sync(0xffffffffu, m.n, 0);
-        const float mean = __shfl_sync(0xffffffffu, m.mean, 0);
-        const float m2 = __shfl_sync(0xffffffffu, m.m2, 0);
-        const float rstd = (float)(1.0 / sqrt((double)m2 / (double)cnt + (double)a.eps));
-        for (int cc = lane; cc < cpg; cc += 32) {
-            const int c = g * cpg + cc;
-            const float sc = a.gamma[c] * rstd;
-            a.scale[(size_t)n * a.C + c] = sc;
-            a.shift[(size_t)n * a.C + c] = a.beta[c] - mean * sc;
-        }
+    for (int i = 0; i < PER; ++i) {
+        const int k = threadIdx.x + i * kGnFinalThreads;
+        p[i] = (k < chunks) ? *(const float4*)(a.partial + (((size_t)n * kGnMaxChunks + k) * a.G + g) * 4)
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    Moments m = {0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < PER; ++i) m = merge(m, Moments{p[i].x, p[i].y, p[i].z});
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        Moments o;
+        o.n = __shfl_down_sync(0xffffffffu, m.n, d);
+        o.mean = __shfl_down_sync(0xffffffffu, m.mean, d);
+        o.m2 = __shfl_down_sync(0xffffffffu, m.m2, d);
+        m = merge(m, o);
+    }
+    if (lane == 0) sm[warp] = m;
+    __syncthreads();
+    Moments t = sm[0];
+#pragma unroll
+    for (int w = 1; w < kGnFinalThreads / 32; ++w) t = merge(t, sm[w]);
+    const float rstd = (float)(1.0 / sqrt((double)t.m2 / (double)t.n + (double)a.eps));
+    for (int cc = threadIdx.x; cc < cpg; cc += kGnFinalThreads) {
+        const int c = g * cpg + cc;
+        const float sc = a.gamma[c] * rstd;
+        a.scale[(size_t)n * a.C + c] = sc;
+        a.shift[(size_t)n * a.C + c] = a.beta[c] - t.mean * sc;
     }
 }
 
@@ -420,7 +428,7 @@ cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s) {
     else gn_partial_kernel<float><<<grid, kGnThreads, 0, s>>>(a, chunks, ppc);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    gn_finalize_kernel<<<a.B, 256, 0, s>>>(a, chunks);
+    gn_finalize_kernel<<<dim3(a.G, a.B), kGnFinalThreads, 0, s>>>(a, chunks);
     return cudaGetLastError();
 }
 

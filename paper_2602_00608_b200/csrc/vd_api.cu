@@ -110,7 +110,8 @@ class Planner {
     // conv step; x at source resolution Hs x Ws
     void add_conv(const std::string& name, const std::vector<std::string>& wnames, int Cout_each, size_t x_off,
                   int in_dtype, int Hs, int Ws, int Cin, int ksize, bool upsample, bool prologue, bool silu,
-                  long residual_off, size_t y_off, int out_dtype, bool out_nchw, bool y_is_frames) {
+                  long residual_off, size_t y_off, int out_dtype, bool out_nchw, bool y_is_frames,
+                  const std::string& shortcut_name = std::string(), size_t x2_off = 0, int Cin2 = 0) {
         Step s{};
         s.kind = VD_STEP_CONV;
         const int Cout = Cout_each * (int)wnames.size();
@@ -124,12 +125,18 @@ class Planner {
         a.B = 0; a.Hs = Hs; a.Ws = Ws; a.H = H; a.W = W;
         a.Cin = Cin; a.Cout = Cout; a.ksize = ksize; a.upsample = upsample; a.silu = silu;
         a.in_dtype = in_dtype; a.out_dtype = out_dtype; a.out_nchw = out_nchw; a.bf16_operands = bf16();
+        if (!shortcut_name.empty()) { a.x2 = ptr<void>(x2_off); a.Cin2 = Cin2; }
         ConvArgs probe = a;
         probe.B = 1;
         const bool tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && conv_tc_supported(probe);
         ConvW cw = conv_weight(wnames, Cout_each, Cin, ksize * ksize, tc);
         a.w = ptr<void>(cw.w_off);
         a.bias = ptr<float>(cw.b_off);
+        if (!shortcut_name.empty()) {          // only requested when the tensor-core kernel takes this layer
+            ConvW sw = conv_weight({shortcut_name}, Cout, Cin2, 1, true);
+            a.w2 = ptr<void>(sw.w_off);
+            a.bias2 = ptr<float>(sw.b_off);
+        }
         s.conv = a;
         s.use_tc = tc;
         s.has_residual = residual_off >= 0;
@@ -139,6 +146,13 @@ class Planner {
         s.info.bytes_per_frame = (double)Hs * Ws * Cin * elt(in_dtype) + P * Cout * elt(out_dtype) +
                                  (residual_off >= 0 ? P * Cout * 4.0 : 0.0);
         s.info.weight_bytes = (double)ksize * ksize * Cin * Cout * elt(cfg_.dtype);
+        s.info.has_residual = residual_off >= 0;
+        if (!shortcut_name.empty()) {
+            s.info.c_in2 = Cin2;
+            s.info.flops_per_frame += 2.0 * Cin2 * (double)Cout * P;
+            s.info.bytes_per_frame += P * Cin2 * 4.0;
+            s.info.weight_bytes += (double)Cin2 * Cout * elt(cfg_.dtype);
+        }
         h_->steps.push_back(s);
     }
 
@@ -161,6 +175,13 @@ class Planner {
         add_gn(p + ".norm2", hbuf_, act_dtype(), H, W, Cout, p + ".norm2");
         long res = (long)x;
         if (Cin != Cout) {
+            const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 64 == 0;
+            if (fuse) {      // the 1x1 shortcut rides along as extra K of conv2: no tensor of its own
+                add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, -1, y,
+                         VD_F32, false, false, p + ".shortcut", x, Cin);
+                cur_x_ ^= 1;
+                return;
+            }
             add_conv(p + ".shortcut", {p + ".shortcut"}, Cout, x, VD_F32, H, W, Cin, 1, false, false, false, -1, sbuf_,
                      VD_F32, false, false);
             res = (long)sbuf_;

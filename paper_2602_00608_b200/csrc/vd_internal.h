@@ -21,6 +21,11 @@ struct ConvArgs {
     int H, W;               // output resolution (= source, or 2x source with upsample)
     int Cin, Cout, ksize, upsample, silu;
     int in_dtype, out_dtype, out_nchw, bf16_operands;
+    // optional fused 1x1 shortcut (tensor-core kernel only): y += W2 * x2 + bias2
+    const void* x2;         // fp32 NHWC [B,H,W,Cin2] at the output resolution, or null
+    const void* w2;         // packed bf16 [Cout][Cin2]
+    const float* bias2;     // [Cout] or null
+    int Cin2;
 };
 
 struct GnArgs {
@@ -78,6 +83,7 @@ cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int 
 // Launch-invariant state of one tensor-core convolution: the TMA descriptor of its packed weights.
 struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
+    unsigned char tmap2[128];   // weights of the fused shortcut (copy of tmap when unused)
     int bn;
     int valid;
 };

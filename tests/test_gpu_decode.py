@@ -158,3 +158,42 @@ def test_decode_argument_errors(env):
     with pytest.raises(vd.VdError) as e:
         vd.Decoder(wl.arch, wl.dtype, 8, 8, 1, wl.groups, wl.eps, bad)
     assert e.value.status == vd.VD_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("flags", [0, 1])
+def test_per_layer_trace_parity(env, flags):
+    """Every block output of the decoder against the oracle's named intermediates (localises an
+    error to a layer): the decode is stopped after each step and that step's output is read back."""
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[2]
+    z = synth.workload_latents(wl, batch=2, h=12, w=20)
+    wts = synth.workload_weights(wl)
+    trace = {}
+    ref.decode(wl.arch, wts, z, wl.groups, wl.eps, trace=trace)
+    dec = vd.Decoder(wl.arch, wl.dtype, 12, 20, 2, wl.groups, wl.eps, wts, flags)
+    zt = torch.from_numpy(z).to("cuda:0", dec.dtype)
+    checked = 0
+    for i, st in enumerate(dec.steps()):
+        name = st["name"]
+        key = None
+        if name in trace:
+            key = name                                     # conv_in, upN.upconv, <block>.conv1, mid.attn.core
+        elif name.endswith(".conv2") and name[:-6] in trace:
+            key = name[:-6]                                # block output (shortcut included)
+        elif name == "mid.attn.o":
+            key = "mid.attn"
+        if key is None or st["out_offset"] < 0:
+            continue
+        dec.stop_after(i)
+        dec.decode(zt)
+        torch.cuda.synchronize()
+        got = dec.read_step_output(st, 2).cpu().numpy()
+        r = rel_l2(got, trace[key])
+        assert r <= 8e-3, (name, r)
+        checked += 1
+    dec.stop_after(-1)
+    assert checked >= 30
+    if flags == 0:
+        impl = {s["name"]: s["impl"] for s in dec.steps()}
+        assert impl["up2.res0.conv2"] == 1 and "up2.res0.shortcut" not in impl      # shortcut fused into conv2
+        assert impl["conv_out"] == 1 and impl["mid.attn.core"] == 1

@@ -185,6 +185,8 @@ TC_CASES = [
     dict(B=1, H=12, W=10, Cin=512, Cout=1536, k=1, upsample=False, prologue=True, silu=False, residual=False, in_bf16=False, out_bf16=True),
     dict(B=1, H=8, W=9, Cin=512, Cout=512, k=1, upsample=False, prologue=False, silu=False, residual=True, in_bf16=True, out_bf16=False),
     dict(B=1, H=17, W=16, Cin=512, Cout=512, k=3, upsample=False, prologue=True, silu=True, residual=True, in_bf16=True, out_bf16=False),
+    dict(B=2, H=37, W=21, Cin=128, Cout=3, k=3, upsample=False, prologue=True, silu=True, residual=False, in_bf16=False, out_bf16=True, out_nchw=True),
+    dict(B=3, H=50, W=70, Cin=128, Cout=128, k=3, upsample=False, prologue=True, silu=True, residual=True, in_bf16=True, out_bf16=False),
 ]
 
 
