@@ -5,11 +5,11 @@
 // each activation crosses HBM once.
 //
 // Persistent kernel, one CTA per SM, roles decoupled through mbarrier rings:
-//   * work item = (16x8-pixel tile, BN-channel block, frame):  D[128 x BN] = sum over taps and
-//     64-channel chunks of A_tap[128 x 64] * W_tap[64 x BN]; CTAs walk the item list with stride
-//     gridDim.x.
-//   * 8 producer warps read the raw 18x10-pixel halo tile of a 64-channel chunk from global
-//     memory once, apply scale/shift (+SiLU), round to bf16 and store it in shared memory in the
+//   * work item = (one or two 16x8-pixel tiles side by side, BN-channel block, frame); per tile
+//     D[128 x BN] = sum over taps and 64-channel chunks of A_tap[128 x 64] * W_tap[64 x BN];
+//     CTAs walk the item list with stride gridDim.x.
+//   * 16 producer warps read the raw halo tile (18 x 10 or 18 x 18 pixels) of a 64-channel chunk
+//     from global memory once (loads of the next batch in flight while this one is transformed), apply scale/shift (+SiLU), round to bf16 and store it in shared memory in the
 //     canonical un-swizzled K-major layout, as eight planes [8 channels][pixel][16 B].  Every tap
 //     is a *view* of that one tile (descriptor start (ky*10+kx) pixels in; eight-row groups are
 //     one tile row = 10 pixels apart), so the transform runs once per element, not once per tap.
@@ -35,34 +35,42 @@ namespace {
 
 using namespace tc;
 
-constexpr int TILE_H = 16, TILE_W = 8;
-constexpr int PH = TILE_H + 2, PW = TILE_W + 2, NPIX = PH * PW;     // 18 x 10 = 180 halo pixels
-constexpr int PLANE = (NPIX + 1) * 16;                               // bytes between 8-channel planes (odd * 16)
-constexpr int A_STAGE_BYTES = 8 * PLANE;                             // one 64-channel chunk (23 168 B)
-constexpr int NUM_PRODUCER_WARPS = 8;
-constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // warps 0-7
-constexpr int EPI_WARP0 = 8;                                         // warps 8-11 (warp % 4 = TMEM lane quarter)
-constexpr int TMA_WARP = 12, MMA_WARP = 13;
-constexpr int NUM_THREADS = 14 * 32;
-constexpr int ITEMS = NPIX * 8;                                      // (pixel, 8-channel group) work items per chunk
+constexpr int TILE_H = 16, TILE_W = 8;                               // one MMA tile: 128 output pixels
+constexpr int PH = TILE_H + 2;
+constexpr int NUM_PRODUCER_WARPS = 16;                               // enough loads in flight to cover DRAM latency
+constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // warps 0-15
+constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
+constexpr int TMA_WARP = 20, MMA_WARP = 21;
+constexpr int NUM_THREADS = 22 * 32;
+constexpr int BATCH = 2;                                             // (pixel, 8-channel) loads per thread per batch
 constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
 
+// BN = output channels per work item; MT = 16x8 MMA tiles per work item (side by side in x) that
+// share every weight stage, which halves the weight traffic through shared memory where the
+// channel block is narrow.
 template <int BN> struct TileCfg {
+    static constexpr int MT = BN == 128 ? 2 : 1;
+    static constexpr int SUPER_W = TILE_W * MT;                      // item width in pixels
+    static constexpr int PW = SUPER_W + 2;                           // halo tile: PH x PW pixels
+    static constexpr int NPIX = PH * PW;
+    static constexpr int PLANE = (NPIX | 1) * 16;                    // bytes between 8-channel planes (odd * 16)
+    static constexpr int A_STAGE_BYTES = 8 * PLANE;                  // one 64-channel chunk of the halo tile
+    static constexpr int ITEMS = NPIX * 8;                           // (pixel, 8-channel group) pairs per chunk
+    static constexpr int NSUB = (ITEMS + NUM_PRODUCERS * BATCH - 1) / (NUM_PRODUCERS * BATCH);
     static constexpr int B_STAGE_BYTES = BN * 128;                   // BN rows x 64 bf16
     static constexpr int B_STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int A_STAGES = BN == 256 ? 3 : 4;
+    static constexpr int A_STAGES = BN == 16 ? 4 : (BN == 128 ? 2 : 3);
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
     static constexpr int SMEM_TOTAL = SMEM_B + SMEM_A + 512 + 1024;  // + barriers + slack for 1024-B alignment
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
-    static constexpr int TMEM_COLS = 2 * ACC_COLS;
+    static constexpr int TMEM_COLS = 2 * MT * ACC_COLS;              // double-buffered
 };
 
 struct Raw8 { uint4 lo, hi; };   // eight channels of one pixel: bf16 -> lo only; fp32 -> lo + hi
 
-template <bool IN_BF16>
-__device__ __forceinline__ void load_raw(const void* x, size_t elem_off, Raw8& r) {
-    if (IN_BF16) {
+__device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t elem_off, Raw8& r) {
+    if (is_bf16) {
         r.lo = __ldg((const uint4*)((const __nv_bfloat16*)x + elem_off));
     } else {
         const float4* p = (const float4*)((const float*)x + elem_off);
@@ -71,9 +79,8 @@ __device__ __forceinline__ void load_raw(const void* x, size_t elem_off, Raw8& r
         r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
     }
 }
-template <bool IN_BF16>
-__device__ __forceinline__ void unpack_raw(const Raw8& r, float v[8]) {
-    if (IN_BF16) {
+__device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[8]) {
+    if (is_bf16) {
         const uint32_t w[4] = {r.lo.x, r.lo.y, r.lo.z, r.lo.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -96,9 +103,9 @@ struct Bars {                    // lives in shared memory
 
 struct Item { int tx0, ty0, n0, b; };
 
-struct Sched {                   // static round-robin over (tile, channel block, frame)
+struct Sched {                   // static round-robin over (item tile, channel block, frame)
     int tiles_x, tiles, nblk, total;
-    __device__ __forceinline__ Item get(int w, int bn) const {
+    __device__ __forceinline__ Item get(int w, int bn, int super_w) const {
         Item it;
         const int per_frame = tiles * nblk;
         it.b = w / per_frame;
@@ -106,7 +113,7 @@ struct Sched {                   // static round-robin over (tile, channel block
         const int t = r / nblk;
         it.n0 = (r - t * nblk) * bn;
         it.ty0 = (t / tiles_x) * TILE_H;
-        it.tx0 = (t % tiles_x) * TILE_W;
+        it.tx0 = (t % tiles_x) * super_w;
         return it;
     }
 };
@@ -117,6 +124,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                unsigned int* status) {
     using Cfg = TileCfg<BN>;
+    constexpr int MT = Cfg::MT, PW = Cfg::PW, PLANE = Cfg::PLANE, ITEMS = Cfg::ITEMS, NSUB = Cfg::NSUB;
+    constexpr int A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* smem_b = smem;
@@ -128,9 +137,10 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     const int taps = a.ksize * a.ksize;
     const int kchunks = a.Cin >> 6;
     const int kchunks2 = a.x2 ? (a.Cin2 >> 6) : 0;          // extra K: 1x1 shortcut on a second input
+    const int ktotal = kchunks + kchunks2;
     const int cout_pad = (a.Cout % 128 == 0) ? a.Cout : 16; // rows per tap in the packed weights
     Sched sched;
-    sched.tiles_x = (a.W + TILE_W - 1) / TILE_W;
+    sched.tiles_x = (a.W + Cfg::SUPER_W - 1) / Cfg::SUPER_W;
     sched.tiles = sched.tiles_x * ((a.H + TILE_H - 1) / TILE_H);
     sched.nblk = cout_pad / BN;
     sched.total = sched.tiles * sched.nblk * a.B;
@@ -151,175 +161,197 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
 
     if (warp < NUM_PRODUCER_WARPS) {
         // ------------------------------------------------ operand prologue (producers)
+        // The work is a flat sequence of batches (item, chunk, sub-batch); the loads of batch n+1
+        // are issued before batch n is transformed, so global-memory latency stays covered.
         const int j = tid & 7;                              // this thread's 8-channel group within a chunk
         const bool prologue = a.scale != nullptr;
         const bool silu = a.silu != 0;
         const int up = a.upsample ? 1 : 0;
+        struct Pos { int w, kc, sub; Item it; };
+        auto advance = [&](Pos& p) {
+            if (++p.sub == NSUB) {
+                p.sub = 0;
+                if (++p.kc == ktotal) {
+                    p.kc = 0;
+                    p.w += gridDim.x;
+                    if (p.w < sched.total) p.it = sched.get(p.w, BN, Cfg::SUPER_W);
+                }
+            }
+        };
+        auto issue = [&](const Pos& p, Raw8 (&raw)[BATCH], uint32_t& vmask) {
+            const bool second = p.kc >= kchunks;
+            const int c0 = (second ? p.kc - kchunks : p.kc) * 64 + j * 8;
+            const bool centre_only = second || a.ksize == 1;
+            vmask = 0;
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int i = (p.sub * BATCH + u) * NUM_PRODUCERS + tid;
+                const int pix = i >> 3;
+                const int py = pix / PW, px = pix - py * PW;
+                const int oy = p.it.ty0 + py - 1, ox = p.it.tx0 + px - 1;
+                bool v = (i < ITEMS) && oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
+                if (centre_only) v = v && py >= 1 && py <= TILE_H && px >= 1 && px <= Cfg::SUPER_W;
+                if (v) {
+                    vmask |= 1u << u;
+                    if (second) load_raw(false, a.x2, (((size_t)p.it.b * a.H + oy) * a.W + ox) * a.Cin2 + c0, raw[u]);
+                    else load_raw(IN_BF16, a.x, (((size_t)p.it.b * a.Hs + (oy >> up)) * a.Ws + (ox >> up)) * a.Cin + c0, raw[u]);
+                }
+            }
+        };
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        constexpr int ITERS = (ITEMS + NUM_PRODUCERS - 1) / NUM_PRODUCERS;          // 6
-        for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x) {
-            const Item it = sched.get(w, BN);
-            const size_t img = (size_t)it.b * a.Hs * a.Ws;
-            for (int kc = 0; kc < kchunks + kchunks2 && ok; ++kc) {
-                const bool second = kc >= kchunks;
-                const int c0 = (second ? kc - kchunks : kc) * 64 + j * 8;
-                float sc[8], sh[8];
-                const bool pro = prologue && !second;
-                if (pro) {
-                    const float4* ps = (const float4*)(a.scale + (size_t)it.b * a.Cin + c0);
-                    const float4* pt = (const float4*)(a.shift + (size_t)it.b * a.Cin + c0);
-                    const float4 s0 = __ldg(ps), s1 = __ldg(ps + 1), t0 = __ldg(pt), t1 = __ldg(pt + 1);
-                    sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
-                    sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
-                }
+        Pos cur;
+        cur.w = blockIdx.x; cur.kc = 0; cur.sub = 0;
+        if (cur.w < sched.total) cur.it = sched.get(cur.w, BN, Cfg::SUPER_W);
+        Raw8 raw_cur[BATCH], raw_next[BATCH];
+        uint32_t vm_cur = 0, vm_next = 0;
+        if (cur.w < sched.total) issue(cur, raw_cur, vm_cur);
+        while (cur.w < sched.total && ok) {
+            Pos nxt = cur;
+            advance(nxt);
+            if (nxt.w < sched.total) issue(nxt, raw_next, vm_next);
+            const bool second = cur.kc >= kchunks;
+            const bool pro = prologue && !second;
+            float sc[8], sh[8];
+            if (pro) {
+                const int c0 = cur.kc * 64 + j * 8;
+                const float4* ps = (const float4*)(a.scale + (size_t)cur.it.b * a.Cin + c0);
+                const float4* pt = (const float4*)(a.shift + (size_t)cur.it.b * a.Cin + c0);
+                const float4 s0 = __ldg(ps), s1 = __ldg(ps + 1), t0 = __ldg(pt), t1 = __ldg(pt + 1);
+                sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
+                sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
+            }
+            if (cur.sub == 0) {
                 ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                 if (!ok) break;
-                uint8_t* dst_plane = smem_a + stage * A_STAGE_BYTES + j * PLANE;
-                const bool centre_only = second || a.ksize == 1;
-                Raw8 raw[ITERS];
-                bool valid[ITERS];
-                if (!second) {
+            }
+            uint8_t* dst_plane = smem_a + stage * A_STAGE_BYTES + j * PLANE;
 #pragma unroll
-                    for (int u = 0; u < ITERS; ++u) {
-                        const int i = u * NUM_PRODUCERS + tid;
-                        const int pix = i >> 3;
-                        const int py = pix / PW, px = pix - py * PW;
-                        const int oy = it.ty0 + py - 1, ox = it.tx0 + px - 1;
-                        bool v = (i < ITEMS) && oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
-                        if (centre_only) v = v && py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
-                        valid[u] = v;
-                        if (v) load_raw<IN_BF16>(a.x, (img + (size_t)(oy >> up) * a.Ws + (ox >> up)) * a.Cin + c0, raw[u]);
-                    }
-                } else {
-                    const size_t img2 = (size_t)it.b * a.H * a.W;
+            for (int u = 0; u < BATCH; ++u) {
+                const int i = (cur.sub * BATCH + u) * NUM_PRODUCERS + tid;
+                if (i >= ITEMS) continue;
+                uint4 out = make_uint4(0u, 0u, 0u, 0u);
+                if (vm_cur & (1u << u)) {
+                    float v[8];
+                    unpack_raw(second ? false : IN_BF16, raw_cur[u], v);
+                    if (pro) {
 #pragma unroll
-                    for (int u = 0; u < ITERS; ++u) {
-                        const int i = u * NUM_PRODUCERS + tid;
-                        const int pix = i >> 3;
-                        const int py = pix / PW, px = pix - py * PW;
-                        const int oy = it.ty0 + py - 1, ox = it.tx0 + px - 1;
-                        const bool v = (i < ITEMS) && oy < a.H && ox < a.W && py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
-                        valid[u] = v;
-                        if (v) load_raw<false>(a.x2, (img2 + (size_t)oy * a.W + ox) * a.Cin2 + c0, raw[u]);
-                    }
-                }
+                        for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
+                        if (silu) {
 #pragma unroll
-                for (int u = 0; u < ITERS; ++u) {
-                    const int i = u * NUM_PRODUCERS + tid;
-                    if (i >= ITEMS) continue;
-                    uint4 out = make_uint4(0u, 0u, 0u, 0u);
-                    if (valid[u]) {
-                        float v[8];
-                        if (second) unpack_raw<false>(raw[u], v);
-                        else unpack_raw<IN_BF16>(raw[u], v);
-                        if (pro) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
-                            if (silu) {
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) v[e] = silu_fast(v[e]);
-                            }
+                            for (int e = 0; e < 8; ++e) v[e] = silu_fast(v[e]);
                         }
-                        out = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
                     }
-                    *(uint4*)(dst_plane + (i >> 3) * 16) = out;
+                    out = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
                 }
+                *(uint4*)(dst_plane + (i >> 3) * 16) = out;
+            }
+            if (cur.sub == NSUB - 1) {
                 fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
                 mbar_arrive(smem_u32(&bars->a_full[stage]));
                 if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
             }
+            cur = nxt;
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) raw_cur[u] = raw_next[u];
+            vm_cur = vm_next;
         }
     } else if (warp < EPI_WARP0 + 4) {
         // ------------------------------------------------ epilogue
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
-        const int m = ew * 32 + lane;                        // accumulator row = pixel of the tile
+        const int m = ew * 32 + lane;                        // accumulator row = pixel of the MMA tile
         bool ok = true;
         int n_item = 0;
         for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x, ++n_item) {
-            const Item it = sched.get(w, BN);
+            const Item it = sched.get(w, BN, Cfg::SUPER_W);
             const int buf = n_item & 1;
             ok = mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item >> 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld below is warp-collective
             if (!ok) break;
             tc_fence_after();
-            const uint32_t tacc = tmem_base + (uint32_t)(buf * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
-            const int oy = it.ty0 + (m >> 3), ox = it.tx0 + (m & 7);
-            const bool inside = oy < a.H && ox < a.W;
-            const size_t opix = ((size_t)it.b * a.H + oy) * a.W + ox;
-            if (OUT_MODE == 2) {
-                uint32_t r[32];
-                tmem_ld32(tacc, r);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars->acc_empty[buf]));
-                if (inside) {
-#pragma unroll
-                    for (int co = 0; co < 16; ++co) {
-                        if (co < a.Cout) {
-                            const float v = __uint_as_float(r[co]) + (a.bias ? __ldg(a.bias + co) : 0.f);
-                            const size_t o = (((size_t)it.b * a.Cout + co) * a.H + oy) * a.W + ox;
-                            if (a.out_dtype == VD_BF16) ((__nv_bfloat16*)a.y)[o] = __float2bfloat16_rn(v);
-                            else ((float*)a.y)[o] = v;
-                        }
-                    }
-                }
-            } else {
-                constexpr int NCB = BN / 32 > 0 ? BN / 32 : 1;
-                const float4* rp = a.residual ? (const float4*)(a.residual + opix * a.Cout + it.n0) : nullptr;
-                float4 res[8];
-                if (rp && inside) {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) res[q] = __ldg(rp + q);
-                }
 #pragma unroll 1
-                for (int cb = 0; cb < NCB; ++cb) {
-                    uint32_t r[32];
-                    tmem_ld32(tacc + (uint32_t)(cb * 32), r);
+            for (int t = 0; t < MT; ++t) {
+                const uint32_t tacc = tmem_base + (uint32_t)((buf * MT + t) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
+                const int oy = it.ty0 + (m >> 3), ox = it.tx0 + t * TILE_W + (m & 7);
+                const bool inside = oy < a.H && ox < a.W;
+                const size_t opix = ((size_t)it.b * a.H + oy) * a.W + ox;
+                const bool last_tile = t == MT - 1;
+                if (OUT_MODE == 2) {
+                    uint32_t r[16];
+                    tmem_ld16(tacc, r);
                     tmem_ld_wait();
-                    if (cb == NCB - 1) {                      // accumulator fully read: hand it back to the MMA warp
+                    if (last_tile) {
                         tc_fence_before();
                         mbar_arrive(smem_u32(&bars->acc_empty[buf]));
                     }
                     if (inside) {
-                        const int co = it.n0 + cb * 32;
-                        float v[32];
 #pragma unroll
-                        for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
-                        if (a.bias) {
-#pragma unroll
-                            for (int q = 0; q < 32; q += 4) {
-                                const float4 t = __ldg((const float4*)(a.bias + co + q));
-                                v[q] += t.x; v[q + 1] += t.y; v[q + 2] += t.z; v[q + 3] += t.w;
+                        for (int co = 0; co < 16; ++co) {
+                            if (co < a.Cout) {
+                                const float v = __uint_as_float(r[co]) + (a.bias ? __ldg(a.bias + co) : 0.f);
+                                const size_t o = (((size_t)it.b * a.Cout + co) * a.H + oy) * a.W + ox;
+                                if (a.out_dtype == VD_BF16) ((__nv_bfloat16*)a.y)[o] = __float2bfloat16_rn(v);
+                                else ((float*)a.y)[o] = v;
                             }
                         }
-                        if (a.bias2) {
+                    }
+                } else {
+                    constexpr int NCB = BN / 16;                  // 16 accumulator columns at a time
+                    const float4* rp = a.residual ? (const float4*)(a.residual + opix * a.Cout + it.n0) : nullptr;
+                    float4 res[4];
+                    if (rp && inside) {
 #pragma unroll
-                            for (int q = 0; q < 32; q += 4) {
-                                const float4 t = __ldg((const float4*)(a.bias2 + co + q));
-                                v[q] += t.x; v[q + 1] += t.y; v[q + 2] += t.z; v[q + 3] += t.w;
-                            }
+                        for (int q = 0; q < 4; ++q) res[q] = __ldg(rp + q);
+                    }
+#pragma unroll 1
+                    for (int cb = 0; cb < NCB; ++cb) {
+                        uint32_t r[16];
+                        tmem_ld16(tacc + (uint32_t)(cb * 16), r);
+                        tmem_ld_wait();
+                        if (last_tile && cb == NCB - 1) {         // accumulators fully read: hand them back to the MMA warp
+                            tc_fence_before();
+                            mbar_arrive(smem_u32(&bars->acc_empty[buf]));
                         }
-                        if (rp) {
+                        if (inside) {
+                            const int co = it.n0 + cb * 16;
+                            float v[16];
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                v[4 * q] += res[q].x; v[4 * q + 1] += res[q].y; v[4 * q + 2] += res[q].z; v[4 * q + 3] += res[q].w;
+                            for (int q = 0; q < 16; ++q) v[q] = __uint_as_float(r[q]);
+                            if (a.bias) {
+#pragma unroll
+                                for (int q = 0; q < 16; q += 4) {
+                                    const float4 tb = __ldg((const float4*)(a.bias + co + q));
+                                    v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
+                                }
                             }
-                            if (cb + 1 < NCB) {               // prefetch the next column block's residual
+                            if (a.bias2) {
 #pragma unroll
-                                for (int q = 0; q < 8; ++q) res[q] = __ldg(rp + (cb + 1) * 8 + q);
+                                for (int q = 0; q < 16; q += 4) {
+                                    const float4 tb = __ldg((const float4*)(a.bias2 + co + q));
+                                    v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
+                                }
                             }
-                        }
-                        if (OUT_MODE == 1) {
-                            uint4* yp = (uint4*)((__nv_bfloat16*)a.y + opix * a.Cout + co);
+                            if (rp) {
 #pragma unroll
-                            for (int q = 0; q < 32; q += 8)
-                                yp[q >> 3] = make_uint4(pack_bf16(v[q], v[q + 1]), pack_bf16(v[q + 2], v[q + 3]),
-                                                        pack_bf16(v[q + 4], v[q + 5]), pack_bf16(v[q + 6], v[q + 7]));
-                        } else {
-                            float4* yp = (float4*)((float*)a.y + opix * a.Cout + co);
+                                for (int q = 0; q < 4; ++q) {
+                                    v[4 * q] += res[q].x; v[4 * q + 1] += res[q].y; v[4 * q + 2] += res[q].z; v[4 * q + 3] += res[q].w;
+                                }
+                                if (cb + 1 < NCB) {               // prefetch the next column block's residual
 #pragma unroll
-                            for (int q = 0; q < 32; q += 4) yp[q >> 2] = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                                    for (int q = 0; q < 4; ++q) res[q] = __ldg(rp + (cb + 1) * 4 + q);
+                                }
+                            }
+                            if (OUT_MODE == 1) {
+                                uint4* yp = (uint4*)((__nv_bfloat16*)a.y + opix * a.Cout + co);
+#pragma unroll
+                                for (int q = 0; q < 16; q += 8)
+                                    yp[q >> 3] = make_uint4(pack_bf16(v[q], v[q + 1]), pack_bf16(v[q + 2], v[q + 3]),
+                                                            pack_bf16(v[q + 4], v[q + 5]), pack_bf16(v[q + 6], v[q + 7]));
+                            } else {
+                                float4* yp = (float4*)((float*)a.y + opix * a.Cout + co);
+#pragma unroll
+                                for (int q = 0; q < 16; q += 4) yp[q >> 2] = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                            }
                         }
                     }
                 }
@@ -332,8 +364,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             int issued = 0;
             bool ok = true;
             for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x) {
-                const Item it = sched.get(w, BN);
-                for (int kc = 0; kc < kchunks + kchunks2 && ok; ++kc) {
+                const Item it = sched.get(w, BN, Cfg::SUPER_W);
+                for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
                     for (int tap = 0; tap < ntap; ++tap) {
@@ -371,8 +403,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 ok = mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item >> 1) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * Cfg::ACC_COLS);
-                for (int kc = 0; kc < kchunks + kchunks2 && ok; ++kc) {
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * MT * Cfg::ACC_COLS);
+                for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
                     ok = mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag);
@@ -385,13 +417,16 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         tc_fence_after();
                         const bool centre = second || a.ksize == 1;
                         const int ky = centre ? 1 : tap / 3, kx = centre ? 1 : tap - 3 * (tap / 3);
-                        const uint32_t a_tap = a_stage + (uint32_t)(ky * PW + kx) * 16;
                         const uint32_t b_stage = smem_u32(smem_b + bs * Cfg::B_STAGE_BYTES);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const uint64_t adesc = make_smem_desc(a_tap + (uint32_t)(2 * k) * PLANE, PLANE, PW * 16, 0);
-                            const uint64_t bdesc = make_smem_desc(b_stage + (uint32_t)k * 32, 16, 1024, 2);
-                            umma_bf16(tmem_d, adesc, bdesc, idesc, (kc | tap | k) != 0);
+                        for (int t = 0; t < MT; ++t) {
+                            const uint32_t a_tap = a_stage + (uint32_t)(ky * PW + kx + t * TILE_W) * 16;
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint64_t adesc = make_smem_desc(a_tap + (uint32_t)(2 * k) * PLANE, PLANE, PW * 16, 0);
+                                const uint64_t bdesc = make_smem_desc(b_stage + (uint32_t)k * 32, 16, 1024, 2);
+                                umma_bf16(tmem_d + (uint32_t)(t * Cfg::ACC_COLS), adesc, bdesc, idesc, (kc | tap | k) != 0);
+                            }
                         }
                         umma_commit(smem_u32(&bars->b_empty[bs]));
                         if (++bs == Cfg::B_STAGES) { bs = 0; bph ^= 1; }
@@ -480,7 +515,7 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int tiles = ((a.W + TILE_W - 1) / TILE_W) * ((a.H + TILE_H - 1) / TILE_H);
+    const int tiles = ((a.W + TileCfg<BN>::SUPER_W - 1) / TileCfg<BN>::SUPER_W) * ((a.H + TILE_H - 1) / TILE_H);
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
     const int grid = (int)std::min<long long>(total, num_sms());
     kern<<<grid, NUM_THREADS, TileCfg<BN>::SMEM_TOTAL, s>>>(a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2, status);
