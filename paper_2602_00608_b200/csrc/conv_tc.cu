@@ -5,23 +5,30 @@
 // each activation crosses HBM once.
 //
 // Persistent kernel, one CTA per SM, roles decoupled through mbarrier rings:
-//   * work item = (one or two 16x8-pixel tiles side by side, BN-channel block, frame); per tile
-//     D[128 x BN] = sum over taps and 64-channel chunks of A_tap[128 x 64] * W_tap[64 x BN];
-//     CTAs walk the item list with stride gridDim.x.
-//   * 16 producer warps read the raw halo tile (18 x 10 or 18 x 18 pixels) of a 64-channel chunk
-//     from global memory once (loads of the next batch in flight while this one is transformed), apply scale/shift (+SiLU), round to bf16 and store it in shared memory in the
-//     canonical un-swizzled K-major layout, as eight planes [8 channels][pixel][16 B].  Every tap
-//     is a *view* of that one tile (descriptor start (ky*10+kx) pixels in; eight-row groups are
-//     one tile row = 10 pixels apart), so the transform runs once per element, not once per tap.
+//   * tile = 16x8 output pixels x BN output channels:  D[128 x BN] = sum over taps and 64-channel
+//     chunks of A_tap[128 x 64] * W_tap[64 x BN].  Every CTA owns a contiguous, balanced range of
+//     tiles and walks it in work items of two tiles that share every weight stage.
+//   * 15 producer warps read the raw 18x10-pixel halo tile of a 64-channel chunk from global
+//     memory once, apply
+//     scale/shift (+SiLU), round to bf16 and store it in shared memory in the canonical
+//     un-swizzled K-major layout, as eight planes [8 channels][pixel][16 B].  Every tap is a *view*
+//     of that one tile (descriptor start (ky*10+kx) pixels in; eight-row groups are one tile row
+//     = 10 pixels apart), so the transform runs once per element, not once per tap.
 //     Out-of-image halo pixels are exact zeros (padding applies to the transformed tensor).
 //     An optional second input (the block's raw input for a width-changing ResNet block) is
 //     appended as extra K with a single centre tap: the 1x1 shortcut without its own round trip.
 //   * 1 warp streams the weights (bf16 [tap][Cout][Cin]) by TMA into 128B-swizzled stages.
-//   * 1 thread issues tcgen05.mma (M=128, N=BN, K=16) into one of two TMEM accumulators.
-//   * 4 epilogue warps drain the other accumulator: tcgen05.ld, + bias (+ fp32 residual,
-//     prefetched one column block ahead), store fp32/bf16 NHWC or the NCHW frame.
+//   * 1 thread issues tcgen05.mma (M=128, N=BN, K=16) into TMEM accumulators (double-buffered
+//     where 4 x BN columns fit).
+//   * 4 epilogue warps drain the accumulators: tcgen05.ld, + bias, and the tile leaves through
+//     shared memory as 128-byte-wide slices written by bulk tensor stores, which coalesce the
+//     traffic and clip the ragged image edge.  Where the layer has a residual, the output buffer
+//     IS the residual stream and the store is a bulk tensor reduce-add (the fp32 add x + conv(h)
+//     is done once, by the memory system), so the residual never passes through the SM.
+//     The 3-channel frame head writes its NCHW planes directly.
 // Every wait is bounded: on expiry the CTA records a code in the status word and unwinds.
 #include <cuda.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -36,45 +43,50 @@ namespace {
 using namespace tc;
 
 constexpr int TILE_H = 16, TILE_W = 8;                               // one MMA tile: 128 output pixels
-constexpr int PH = TILE_H + 2;
-constexpr int NUM_PRODUCER_WARPS = 16;                               // enough loads in flight to cover DRAM latency
-constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // warps 0-15
+constexpr int PH = TILE_H + 2, PW = TILE_W + 2, NPIX = PH * PW;     // 18 x 10 = 180 halo pixels
+constexpr int PLANE = (NPIX + 1) * 16;                               // bytes between 8-channel planes (odd * 16)
+constexpr int A_TILE_BYTES = 8 * PLANE;                              // one 64-channel chunk of one tile (23 168 B)
+constexpr int ITEMS = NPIX * 8;                                      // (pixel, 8-channel group) pairs per tile chunk
+constexpr int NUM_PRODUCER_WARPS = 15;
+constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // 480 = ITEMS / 3: three pairs per thread
+constexpr int BATCH = ITEMS / NUM_PRODUCERS;                         // 3
+static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the halo chunk exactly");
+constexpr int TMA_WARP = 15;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
-constexpr int TMA_WARP = 20, MMA_WARP = 21;
-constexpr int NUM_THREADS = 22 * 32;
-constexpr int BATCH = 2;                                             // (pixel, 8-channel) loads per thread per batch
+constexpr int MMA_WARP = 20;
+constexpr int NUM_THREADS = 21 * 32;
 constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
+constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixels x 128 B: one output slice in smem
 
-// BN = output channels per work item; MT = 16x8 MMA tiles per work item (side by side in x) that
-// share every weight stage, which halves the weight traffic through shared memory where the
-// channel block is narrow.
+// BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
+// item is two 16x8-pixel tiles whose MMAs consume every weight stage together, which halves the
+// weight traffic through shared memory and the bytes the TMA pipeline must keep in flight.
 template <int BN> struct TileCfg {
-    static constexpr int MT = BN == 128 ? 2 : 1;
-    static constexpr int SUPER_W = TILE_W * MT;                      // item width in pixels
-    static constexpr int PW = SUPER_W + 2;                           // halo tile: PH x PW pixels
-    static constexpr int NPIX = PH * PW;
-    static constexpr int PLANE = (NPIX | 1) * 16;                    // bytes between 8-channel planes (odd * 16)
-    static constexpr int A_STAGE_BYTES = 8 * PLANE;                  // one 64-channel chunk of the halo tile
-    static constexpr int ITEMS = NPIX * 8;                           // (pixel, 8-channel group) pairs per chunk
-    static constexpr int NSUB = (ITEMS + NUM_PRODUCERS * BATCH - 1) / (NUM_PRODUCERS * BATCH);
+    static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item
     static constexpr int B_STAGE_BYTES = BN * 128;                   // BN rows x 64 bf16
     static constexpr int B_STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int A_STAGES = BN == 16 ? 4 : (BN == 128 ? 2 : 3);
+    static constexpr int A_STAGES = 2;
+    static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
+    static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
-    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_A + 512 + 1024;  // + barriers + slack for 1024-B alignment
+    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + 512 + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
-    static constexpr int TMEM_COLS = 2 * MT * ACC_COLS;              // double-buffered
+    static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
+    static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
 };
 
 struct Raw8 { uint4 lo, hi; };   // eight channels of one pixel: bf16 -> lo only; fp32 -> lo + hi
 
-__device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t elem_off, Raw8& r) {
+// bf16: the thread's 16 bytes are channels [8j, 8j+8) of the chunk.  fp32: two 16-byte loads,
+// channels [4j, 4j+4) and [32+4j, 32+4j+4), so that the eight threads of a pixel read two
+// contiguous 128-byte lines.
+__device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix_off, int c0, int j, Raw8& r) {
     if (is_bf16) {
-        r.lo = __ldg((const uint4*)((const __nv_bfloat16*)x + elem_off));
+        r.lo = __ldg((const uint4*)((const __nv_bfloat16*)x + pix_off + c0 + j * 8));
     } else {
-        const float4* p = (const float4*)((const float*)x + elem_off);
-        const float4 a = __ldg(p), b = __ldg(p + 1);
+        const float* p = (const float*)x + pix_off + c0 + j * 4;
+        const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 32));
         r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
         r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
     }
@@ -97,40 +109,49 @@ struct Bars {                    // lives in shared memory
     uint64_t a_full[MAX_A_STAGES], a_empty[MAX_A_STAGES];
     uint64_t b_full[MAX_B_STAGES], b_empty[MAX_B_STAGES];
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t epi_sync;           // rendezvous of the 128 epilogue threads (a bounded stand-in for bar.sync)
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
 
-struct Item { int tx0, ty0, n0, b; };
+struct Tile { int tx0, ty0, n0, b; };
 
-struct Sched {                   // static round-robin over (item tile, channel block, frame)
+// Tiles are numbered (frame, channel block, tile row, tile column), column fastest.  Every CTA
+// owns a contiguous, balanced range of tile numbers and walks it in items of `pair` tiles (one
+// when the range or the channel block ends).
+struct Sched {
     int tiles_x, tiles, nblk, total;
-    __device__ __forceinline__ Item get(int w, int bn, int super_w) const {
-        Item it;
-        const int per_frame = tiles * nblk;
-        it.b = w / per_frame;
-        const int r = w - it.b * per_frame;
-        const int t = r / nblk;
-        it.n0 = (r - t * nblk) * bn;
-        it.ty0 = (t / tiles_x) * TILE_H;
-        it.tx0 = (t % tiles_x) * super_w;
-        return it;
+    int begin, end, pair;
+    __device__ __forceinline__ Tile get(int t, int bn) const {
+        Tile r;
+        const int blk = t / tiles;               // frame * nblk + channel block
+        const int s = t - blk * tiles;
+        r.b = blk / nblk;
+        r.n0 = (blk - r.b * nblk) * bn;
+        r.ty0 = (s / tiles_x) * TILE_H;
+        r.tx0 = (s % tiles_x) * TILE_W;
+        return r;
+    }
+    // number of tiles of the item that starts at tile t
+    __device__ __forceinline__ int count(int t) const {
+        return (pair == 2 && t + 1 < end && (t + 1) / tiles == t / tiles) ? 2 : 1;
     }
 };
 
-// OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC, 2 = NCHW frame (dtype from a.out_dtype)
+// OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC (both through shared memory and TMA stores),
+//           2 = NCHW frame written directly (dtype from a.out_dtype)
 template <int BN, bool IN_BF16, int OUT_MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
-               unsigned int* status) {
+               const __grid_constant__ CUtensorMap tmap_y, unsigned int* status) {
     using Cfg = TileCfg<BN>;
-    constexpr int MT = Cfg::MT, PW = Cfg::PW, PLANE = Cfg::PLANE, ITEMS = Cfg::ITEMS, NSUB = Cfg::NSUB;
-    constexpr int A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
+    constexpr int NBUF = Cfg::NBUF, PAIR = Cfg::PAIR, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* smem_b = smem;
-    uint8_t* smem_a = smem + Cfg::SMEM_B;
-    Bars* bars = (Bars*)(smem + Cfg::SMEM_B + Cfg::SMEM_A);
+    uint8_t* smem_out = smem + Cfg::SMEM_B;
+    uint8_t* smem_a = smem_out + Cfg::SMEM_OUT;
+    Bars* bars = (Bars*)(smem_a + Cfg::SMEM_A);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -140,15 +161,19 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     const int ktotal = kchunks + kchunks2;
     const int cout_pad = (a.Cout % 128 == 0) ? a.Cout : 16; // rows per tap in the packed weights
     Sched sched;
-    sched.tiles_x = (a.W + Cfg::SUPER_W - 1) / Cfg::SUPER_W;
+    sched.tiles_x = (a.W + TILE_W - 1) / TILE_W;
     sched.tiles = sched.tiles_x * ((a.H + TILE_H - 1) / TILE_H);
     sched.nblk = cout_pad / BN;
     sched.total = sched.tiles * sched.nblk * a.B;
+    sched.begin = (int)(((long long)sched.total * blockIdx.x) / gridDim.x);
+    sched.end = (int)(((long long)sched.total * (blockIdx.x + 1)) / gridDim.x);
+    sched.pair = PAIR;
 
     if (tid == 0) {
-        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCERS); mbar_init(smem_u32(&bars->a_empty[i]), 1); }
+        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), 1); }
         for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 128); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
+        mbar_init(smem_u32(&bars->epi_sync), 128);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -161,79 +186,72 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
 
     if (warp < NUM_PRODUCER_WARPS) {
         // ------------------------------------------------ operand prologue (producers)
-        // The work is a flat sequence of batches (item, chunk, sub-batch); the loads of batch n+1
-        // are issued before batch n is transformed, so global-memory latency stays covered.
-        const int j = tid & 7;                              // this thread's 8-channel group within a chunk
+        // The work is a flat sequence of units (item, chunk, tile slot); a unit's loads (three
+        // 8-channel groups per thread, 480 threads) are all in flight before any is consumed.
+        const int j = tid & 7;                              // this thread's channel group within a chunk
         const bool prologue = a.scale != nullptr;
         const bool silu = a.silu != 0;
         const int up = a.upsample ? 1 : 0;
-        struct Pos { int w, kc, sub; Item it; };
+        struct Pos { int t, cnt, kc, slot; Tile tile; };
         auto advance = [&](Pos& p) {
-            if (++p.sub == NSUB) {
-                p.sub = 0;
+            if (++p.slot == p.cnt) {
+                p.slot = 0;
                 if (++p.kc == ktotal) {
                     p.kc = 0;
-                    p.w += gridDim.x;
-                    if (p.w < sched.total) p.it = sched.get(p.w, BN, Cfg::SUPER_W);
+                    p.t += p.cnt;
+                    if (p.t < sched.end) p.cnt = sched.count(p.t);
                 }
             }
-        };
-        auto issue = [&](const Pos& p, Raw8 (&raw)[BATCH], uint32_t& vmask) {
-            const bool second = p.kc >= kchunks;
-            const int c0 = (second ? p.kc - kchunks : p.kc) * 64 + j * 8;
-            const bool centre_only = second || a.ksize == 1;
-            vmask = 0;
-#pragma unroll
-            for (int u = 0; u < BATCH; ++u) {
-                const int i = (p.sub * BATCH + u) * NUM_PRODUCERS + tid;
-                const int pix = i >> 3;
-                const int py = pix / PW, px = pix - py * PW;
-                const int oy = p.it.ty0 + py - 1, ox = p.it.tx0 + px - 1;
-                bool v = (i < ITEMS) && oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
-                if (centre_only) v = v && py >= 1 && py <= TILE_H && px >= 1 && px <= Cfg::SUPER_W;
-                if (v) {
-                    vmask |= 1u << u;
-                    if (second) load_raw(false, a.x2, (((size_t)p.it.b * a.H + oy) * a.W + ox) * a.Cin2 + c0, raw[u]);
-                    else load_raw(IN_BF16, a.x, (((size_t)p.it.b * a.Hs + (oy >> up)) * a.Ws + (ox >> up)) * a.Cin + c0, raw[u]);
-                }
-            }
+            if (p.t < sched.end) p.tile = sched.get(p.t + p.slot, BN);
         };
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         Pos cur;
-        cur.w = blockIdx.x; cur.kc = 0; cur.sub = 0;
-        if (cur.w < sched.total) cur.it = sched.get(cur.w, BN, Cfg::SUPER_W);
-        Raw8 raw_cur[BATCH], raw_next[BATCH];
-        uint32_t vm_cur = 0, vm_next = 0;
-        if (cur.w < sched.total) issue(cur, raw_cur, vm_cur);
-        while (cur.w < sched.total && ok) {
-            Pos nxt = cur;
-            advance(nxt);
-            if (nxt.w < sched.total) issue(nxt, raw_next, vm_next);
+        cur.t = sched.begin; cur.kc = 0; cur.slot = 0; cur.cnt = 1;
+        if (cur.t < sched.end) { cur.cnt = sched.count(cur.t); cur.tile = sched.get(cur.t, BN); }
+        while (cur.t < sched.end && ok) {
             const bool second = cur.kc >= kchunks;
+            const bool in_bf16 = second ? false : IN_BF16;
+            const int c0 = (second ? cur.kc - kchunks : cur.kc) * 64;
+            const bool centre_only = second || a.ksize == 1;
+            Raw8 raw[BATCH];
+            uint32_t vm = 0;
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int pix = (u * NUM_PRODUCERS + tid) >> 3;
+                const int py = pix / PW, px = pix - py * PW;
+                const int oy = cur.tile.ty0 + py - 1, ox = cur.tile.tx0 + px - 1;
+                bool v = oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
+                if (centre_only) v = v && py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
+                if (v) {
+                    vm |= 1u << u;
+                    if (second) load_raw(false, a.x2, (((size_t)cur.tile.b * a.H + oy) * a.W + ox) * a.Cin2, c0, j, raw[u]);
+                    else load_raw(IN_BF16, a.x, (((size_t)cur.tile.b * a.Hs + (oy >> up)) * a.Ws + (ox >> up)) * a.Cin, c0, j, raw[u]);
+                }
+            }
             const bool pro = prologue && !second;
             float sc[8], sh[8];
             if (pro) {
-                const int c0 = cur.kc * 64 + j * 8;
-                const float4* ps = (const float4*)(a.scale + (size_t)cur.it.b * a.Cin + c0);
-                const float4* pt = (const float4*)(a.shift + (size_t)cur.it.b * a.Cin + c0);
-                const float4 s0 = __ldg(ps), s1 = __ldg(ps + 1), t0 = __ldg(pt), t1 = __ldg(pt + 1);
+                // channels of v[0..3] and v[4..7] (see load_raw)
+                const int ca = c0 + (in_bf16 ? j * 8 : j * 4), cb = in_bf16 ? ca + 4 : ca + 32;
+                const float* ps = a.scale + (size_t)cur.tile.b * a.Cin;
+                const float* pt = a.shift + (size_t)cur.tile.b * a.Cin;
+                const float4 s0 = __ldg((const float4*)(ps + ca)), s1 = __ldg((const float4*)(ps + cb));
+                const float4 t0 = __ldg((const float4*)(pt + ca)), t1 = __ldg((const float4*)(pt + cb));
                 sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
                 sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
             }
-            if (cur.sub == 0) {
+            if (cur.slot == 0) {
                 ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                 if (!ok) break;
             }
-            uint8_t* dst_plane = smem_a + stage * A_STAGE_BYTES + j * PLANE;
+            uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur.slot * A_TILE_BYTES;
 #pragma unroll
             for (int u = 0; u < BATCH; ++u) {
-                const int i = (cur.sub * BATCH + u) * NUM_PRODUCERS + tid;
-                if (i >= ITEMS) continue;
-                uint4 out = make_uint4(0u, 0u, 0u, 0u);
-                if (vm_cur & (1u << u)) {
+                uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
+                if (vm & (1u << u)) {
                     float v[8];
-                    unpack_raw(second ? false : IN_BF16, raw_cur[u], v);
+                    unpack_raw(in_bf16, raw[u], v);
                     if (pro) {
 #pragma unroll
                         for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
@@ -242,129 +260,149 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             for (int e = 0; e < 8; ++e) v[e] = silu_fast(v[e]);
                         }
                     }
-                    out = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+                    o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]);
                 }
-                *(uint4*)(dst_plane + (i >> 3) * 16) = out;
+                const int pix = (u * NUM_PRODUCERS + tid) >> 3;
+                if (in_bf16) {
+                    *(uint4*)(dst_tile + j * PLANE + pix * 16) = make_uint4(o0, o1, o2, o3);
+                } else {     // channels 4j..4j+3 -> plane j/2, half j&1; channels 32+4j.. -> plane 4 + j/2
+                    uint8_t* q = dst_tile + (j >> 1) * PLANE + pix * 16 + (j & 1) * 8;
+                    *(uint2*)q = make_uint2(o0, o1);
+                    *(uint2*)(q + 4 * PLANE) = make_uint2(o2, o3);
+                }
             }
-            if (cur.sub == NSUB - 1) {
+            if (cur.slot == cur.cnt - 1) {
                 fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
-                mbar_arrive(smem_u32(&bars->a_full[stage]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[stage]));
                 if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
             }
-            cur = nxt;
-#pragma unroll
-            for (int u = 0; u < BATCH; ++u) raw_cur[u] = raw_next[u];
-            vm_cur = vm_next;
+            advance(cur);
         }
-    } else if (warp < EPI_WARP0 + 4) {
+    } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------ epilogue
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
         const int m = ew * 32 + lane;                        // accumulator row = pixel of the MMA tile
+        const bool leader = warp == EPI_WARP0 && lane == 0;  // issues the bulk stores
+        const bool accumulate = a.residual != nullptr;       // y already holds the residual: add into it
         bool ok = true;
         int n_item = 0;
-        for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x, ++n_item) {
-            const Item it = sched.get(w, BN, Cfg::SUPER_W);
-            const int buf = n_item & 1;
-            ok = mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item >> 1) & 1, abort_flag);
+        uint32_t n_slice = 0, sync_phase = 0;
+        auto epi_rendezvous = [&]() {                        // all 128 epilogue threads meet here; bounded like every wait
+            mbar_arrive(smem_u32(&bars->epi_sync));
+            const bool r = mbar_wait(smem_u32(&bars->epi_sync), sync_phase, abort_flag);
+            sync_phase ^= 1;
+            return r;
+        };
+        for (int t = sched.begin; t < sched.end && ok; ++n_item) {
+            const int cnt = sched.count(t);
+            const int buf = n_item % NBUF;
+            ok = mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld below is warp-collective
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
-            for (int t = 0; t < MT; ++t) {
-                const uint32_t tacc = tmem_base + (uint32_t)((buf * MT + t) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
-                const int oy = it.ty0 + (m >> 3), ox = it.tx0 + t * TILE_W + (m & 7);
-                const bool inside = oy < a.H && ox < a.W;
-                const size_t opix = ((size_t)it.b * a.H + oy) * a.W + ox;
-                const bool last_tile = t == MT - 1;
+            for (int slot = 0; slot < cnt; ++slot) {
+                const Tile tl = sched.get(t + slot, BN);
+                const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
+                const bool last_tile = slot == cnt - 1;
                 if (OUT_MODE == 2) {
+                    const int oy = tl.ty0 + (m >> 3), ox = tl.tx0 + (m & 7);
                     uint32_t r[16];
                     tmem_ld16(tacc, r);
                     tmem_ld_wait();
                     if (last_tile) {
                         tc_fence_before();
-                        mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
                     }
-                    if (inside) {
+                    if (oy < a.H && ox < a.W) {
 #pragma unroll
                         for (int co = 0; co < 16; ++co) {
                             if (co < a.Cout) {
                                 const float v = __uint_as_float(r[co]) + (a.bias ? __ldg(a.bias + co) : 0.f);
-                                const size_t o = (((size_t)it.b * a.Cout + co) * a.H + oy) * a.W + ox;
+                                const size_t o = (((size_t)tl.b * a.Cout + co) * a.H + oy) * a.W + ox;
                                 if (a.out_dtype == VD_BF16) ((__nv_bfloat16*)a.y)[o] = __float2bfloat16_rn(v);
                                 else ((float*)a.y)[o] = v;
                             }
                         }
                     }
                 } else {
-                    constexpr int NCB = BN / 16;                  // 16 accumulator columns at a time
-                    const float4* rp = a.residual ? (const float4*)(a.residual + opix * a.Cout + it.n0) : nullptr;
-                    float4 res[4];
-                    if (rp && inside) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) res[q] = __ldg(rp + q);
-                    }
+                    // The tile leaves through shared memory in 128-byte-wide slices (32 fp32 or 64
+                    // bf16 channels), written row-per-thread in the 128B-swizzled layout a bulk
+                    // tensor store expects; the store clips the ragged image edge by itself.
+                    constexpr int CS = OUT_MODE == 0 ? 32 : 64;       // channels per slice
+                    constexpr int NS = BN / CS;
 #pragma unroll 1
-                    for (int cb = 0; cb < NCB; ++cb) {
-                        uint32_t r[16];
-                        tmem_ld16(tacc + (uint32_t)(cb * 16), r);
-                        tmem_ld_wait();
-                        if (last_tile && cb == NCB - 1) {         // accumulators fully read: hand them back to the MMA warp
-                            tc_fence_before();
-                            mbar_arrive(smem_u32(&bars->acc_empty[buf]));
-                        }
-                        if (inside) {
-                            const int co = it.n0 + cb * 16;
-                            float v[16];
+                    for (int sidx = 0; sidx < NS; ++sidx, ++n_slice) {
+                        uint8_t* obuf = smem_out + (n_slice & 1) * OUT_SLICE_BYTES;
+                        if (leader) bulk_wait_group_read<1>();        // the store that last read this buffer is done
+                        ok = __all_sync(0xffffffffu, epi_rendezvous());
+                        if (!ok) break;
+                        uint8_t* orow = obuf + m * 128;
 #pragma unroll
-                            for (int q = 0; q < 16; ++q) v[q] = __uint_as_float(r[q]);
+                        for (int h = 0; h < CS / 32; ++h) {
+                            uint32_t r[32];
+                            tmem_ld32(tacc + (uint32_t)(sidx * CS + h * 32), r);
+                            tmem_ld_wait();
+                            if (last_tile && sidx == NS - 1 && h == CS / 32 - 1) {   // accumulators fully read
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                            }
+                            const int co = tl.n0 + sidx * CS + h * 32;
+                            float v[32];
+#pragma unroll
+                            for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
                             if (a.bias) {
 #pragma unroll
-                                for (int q = 0; q < 16; q += 4) {
+                                for (int q = 0; q < 32; q += 4) {
                                     const float4 tb = __ldg((const float4*)(a.bias + co + q));
                                     v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
                                 }
                             }
                             if (a.bias2) {
 #pragma unroll
-                                for (int q = 0; q < 16; q += 4) {
+                                for (int q = 0; q < 32; q += 4) {
                                     const float4 tb = __ldg((const float4*)(a.bias2 + co + q));
                                     v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
                                 }
                             }
-                            if (rp) {
+                            if (OUT_MODE == 0) {
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    v[4 * q] += res[q].x; v[4 * q + 1] += res[q].y; v[4 * q + 2] += res[q].z; v[4 * q + 3] += res[q].w;
-                                }
-                                if (cb + 1 < NCB) {               // prefetch the next column block's residual
-#pragma unroll
-                                    for (int q = 0; q < 4; ++q) res[q] = __ldg(rp + (cb + 1) * 4 + q);
-                                }
-                            }
-                            if (OUT_MODE == 1) {
-                                uint4* yp = (uint4*)((__nv_bfloat16*)a.y + opix * a.Cout + co);
-#pragma unroll
-                                for (int q = 0; q < 16; q += 8)
-                                    yp[q >> 3] = make_uint4(pack_bf16(v[q], v[q + 1]), pack_bf16(v[q + 2], v[q + 3]),
-                                                            pack_bf16(v[q + 4], v[q + 5]), pack_bf16(v[q + 6], v[q + 7]));
+                                for (int c = 0; c < 8; ++c)
+                                    *(float4*)(orow + ((c ^ (m & 7)) << 4)) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
                             } else {
-                                float4* yp = (float4*)((float*)a.y + opix * a.Cout + co);
 #pragma unroll
-                                for (int q = 0; q < 16; q += 4) yp[q >> 2] = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                                for (int c = 0; c < 4; ++c)
+                                    *(uint4*)(orow + (((h * 4 + c) ^ (m & 7)) << 4)) =
+                                        make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
+                                                   pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
                             }
                         }
+                        fence_proxy_async_smem();
+                        ok = __all_sync(0xffffffffu, epi_rendezvous());
+                        if (!ok) break;
+                        if (leader) {
+                            if (accumulate) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sidx * CS, tl.tx0, tl.ty0, tl.b);
+                            else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sidx * CS, tl.tx0, tl.ty0, tl.b);
+                            bulk_commit_group();
+                        }
                     }
+                    if (!ok) break;
                 }
             }
+            t += cnt;
         }
+        if (leader) bulk_wait_group<0>();                    // all stores have landed before the CTA retires
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x) {
-                const Item it = sched.get(w, BN, Cfg::SUPER_W);
+            for (int t = sched.begin; t < sched.end && ok; t += sched.count(t)) {
+                const Tile tl = sched.get(t, BN);
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
@@ -373,8 +411,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         if (!ok) break;
                         const uint32_t full = smem_u32(&bars->b_full[stage]);
                         mbar_arrive_expect_tx(full, Cfg::B_STAGE_BYTES);
-                        if (second) tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap2, (kc - kchunks) * 64, it.n0, full);
-                        else tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap, kc * 64, tap * cout_pad + it.n0, full);
+                        if (second) tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap2, (kc - kchunks) * 64, tl.n0, full);
+                        else tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap, kc * 64, tap * cout_pad + tl.n0, full);
                         ++issued;
                         if (++stage == Cfg::B_STAGES) { stage = 0; phase ^= 1; }
                     }
@@ -391,19 +429,20 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
             }
         }
-    } else {
+    } else if (warp == MMA_WARP) {
         // ------------------------------------------------ MMA issue
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_bf16(128, BN);
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
             bool ok = true;
             int n_item = 0;
-            for (int w = blockIdx.x; w < sched.total && ok; w += gridDim.x, ++n_item) {
-                const int buf = n_item & 1;
-                ok = mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item >> 1) & 1) ^ 1, abort_flag);
+            for (int t = sched.begin; t < sched.end && ok; ++n_item) {
+                const int cnt = sched.count(t);
+                const int buf = n_item % NBUF;
+                ok = mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * MT * Cfg::ACC_COLS);
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
@@ -418,14 +457,13 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const bool centre = second || a.ksize == 1;
                         const int ky = centre ? 1 : tap / 3, kx = centre ? 1 : tap - 3 * (tap / 3);
                         const uint32_t b_stage = smem_u32(smem_b + bs * Cfg::B_STAGE_BYTES);
-#pragma unroll
-                        for (int t = 0; t < MT; ++t) {
-                            const uint32_t a_tap = a_stage + (uint32_t)(ky * PW + kx + t * TILE_W) * 16;
+                        for (int slot = 0; slot < cnt; ++slot) {
+                            const uint32_t a_tap = a_stage + (uint32_t)(slot * A_TILE_BYTES) + (uint32_t)(ky * PW + kx) * 16;
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
                                 const uint64_t adesc = make_smem_desc(a_tap + (uint32_t)(2 * k) * PLANE, PLANE, PW * 16, 0);
                                 const uint64_t bdesc = make_smem_desc(b_stage + (uint32_t)k * 32, 16, 1024, 2);
-                                umma_bf16(tmem_d + (uint32_t)(t * Cfg::ACC_COLS), adesc, bdesc, idesc, (kc | tap | k) != 0);
+                                umma_bf16(tmem_d + (uint32_t)(slot * Cfg::ACC_COLS), adesc, bdesc, idesc, (kc | tap | k) != 0);
                             }
                         }
                         umma_commit(smem_u32(&bars->b_empty[bs]));
@@ -435,6 +473,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
                 if (ok) umma_commit(smem_u32(&bars->acc_full[buf]));
+                t += cnt;
             }
         }
     }
@@ -515,10 +554,11 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int tiles = ((a.W + TileCfg<BN>::SUPER_W - 1) / TileCfg<BN>::SUPER_W) * ((a.H + TILE_H - 1) / TILE_H);
+    const int tiles = ((a.W + TILE_W - 1) / TILE_W) * ((a.H + TILE_H - 1) / TILE_H);
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
     const int grid = (int)std::min<long long>(total, num_sms());
-    kern<<<grid, NUM_THREADS, TileCfg<BN>::SMEM_TOTAL, s>>>(a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2, status);
+    kern<<<grid, NUM_THREADS, TileCfg<BN>::SMEM_TOTAL, s>>>(a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
+                                                            *(const CUtensorMap*)plan.tmap_y, status);
     return cudaGetLastError();
 }
 
@@ -561,13 +601,34 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     } else {
         memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
     }
+    if (!a.out_nchw) {
+        // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one 128-byte-wide slice of a tile
+        EncodeTiledFn enc = get_encode_fn();
+        if (!enc) return cudaErrorNotSupported;
+        const bool ob = a.out_dtype == VD_BF16;
+        const cuuint64_t es = ob ? 2 : 4;
+        const cuuint64_t dims[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)std::max(a.B, 1)};
+        const cuuint64_t strides[3] = {(cuuint64_t)a.Cout * es, (cuuint64_t)a.W * a.Cout * es, (cuuint64_t)a.H * a.W * a.Cout * es};
+        const cuuint32_t box[4] = {ob ? 64u : 32u, (cuuint32_t)TILE_W, (cuuint32_t)TILE_H, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc((CUtensorMap*)plan->tmap_y, ob ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.y, dims,
+                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    } else {
+        memcpy(plan->tmap_y, plan->tmap, sizeof(plan->tmap));
+    }
     plan->bn = bn;
+    plan->batch = a.B;
+    plan->y = a.y;
     plan->valid = 1;
     return cudaSuccess;
 }
 
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
     if (!plan.valid) return cudaErrorInvalidValue;
+    if (!a.out_nchw && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
+    if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2>(a, plan, status, s) : launch_one<16, false, 2>(a, plan, status, s);

@@ -173,26 +173,27 @@ class Planner {
         add_conv(p + ".conv1", {p + ".conv1"}, Cout, x, VD_F32, H, W, Cin, 3, false, true, true, -1, hbuf_, act_dtype(),
                  false, false);
         add_gn(p + ".norm2", hbuf_, act_dtype(), H, W, Cout, p + ".norm2");
-        long res = (long)x;
-        if (Cin != Cout) {
-            const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 64 == 0;
-            if (fuse) {      // the 1x1 shortcut rides along as extra K of conv2: no tensor of its own
-                add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, -1, y,
-                         VD_F32, false, false, p + ".shortcut", x, Cin);
-                cur_x_ ^= 1;
-                return;
-            }
-            add_conv(p + ".shortcut", {p + ".shortcut"}, Cout, x, VD_F32, H, W, Cin, 1, false, false, false, -1, sbuf_,
+        if (Cin == Cout) {
+            // identity skip: conv2 accumulates into the residual stream in place (x += conv2(...))
+            add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, (long)x, x,
                      VD_F32, false, false);
-            res = (long)sbuf_;
+            return;
         }
-        add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, res, y,
-                 VD_F32, false, false);
+        const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 64 == 0;
+        if (fuse) {      // the 1x1 shortcut rides along as extra K of conv2: no tensor of its own
+            add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, -1, y,
+                     VD_F32, false, false, p + ".shortcut", x, Cin);
+        } else {
+            add_conv(p + ".shortcut", {p + ".shortcut"}, Cout, x, VD_F32, H, W, Cin, 1, false, false, false, -1, y, VD_F32,
+                     false, false);
+            add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, (long)y, y,
+                     VD_F32, false, false);
+        }
         cur_x_ ^= 1;
     }
 
     void attention(const std::string& p, int C, int H, int W) {
-        const size_t x = xs_[cur_x_], y = xs_[cur_x_ ^ 1];
+        const size_t x = xs_[cur_x_];
         add_gn(p + ".norm", x, VD_F32, H, W, C, p + ".norm");
         add_conv(p + ".qkv", {p + ".q", p + ".k", p + ".v"}, C, x, VD_F32, H, W, C, 1, false, true, false, -1, qkv_,
                  act_dtype(), false, false);
@@ -207,9 +208,8 @@ class Planner {
         s.info.flops_per_frame = 4.0 * T * T * C;
         s.info.bytes_per_frame = 4.0 * T * C * es;
         h_->steps.push_back(s);
-        add_conv(p + ".o", {p + ".o"}, C, attno_, act_dtype(), H, W, C, 1, false, false, false, (long)x, y, VD_F32,
-                 false, false);
-        cur_x_ ^= 1;
+        add_conv(p + ".o", {p + ".o"}, C, attno_, act_dtype(), H, W, C, 1, false, false, false, (long)x, x, VD_F32,
+                 false, false);          // x += Wo o + bo, in place
     }
 
     void upconv(const std::string& p, int Cin, int Cout, int Hs, int Ws) {
@@ -259,7 +259,6 @@ class Planner {
         xs_[0] = alloc((size_t)B * max_x * 4);
         xs_[1] = alloc((size_t)B * max_x * 4);
         hbuf_ = alloc((size_t)B * max_h * ae);
-        sbuf_ = max_s ? alloc((size_t)B * max_s * 4) : 0;
         qkv_ = qkv ? alloc((size_t)B * qkv * ae) : 0;
         attno_ = ao ? alloc((size_t)B * ao * ae) : 0;
         vt_ = ao ? alloc(attn_tc_scratch_bytes(B, (int)P0, 512)) : 0;
@@ -328,7 +327,7 @@ class Planner {
     char* base_;
     const vd_config& cfg_;
     size_t cur_ = 0;
-    size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, sbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
+    size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
     int cur_x_ = 0;
 };
@@ -508,7 +507,9 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
     }
     for (Step& st : h->steps) {
         if (st.kind == VD_STEP_CONV && st.use_tc) {
-            e = conv_tc_prepare(st.conv, &st.tc);
+            ConvArgs pa = st.conv;
+            pa.B = cfg->max_batch;
+            e = conv_tc_prepare(pa, &st.tc);
             if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "weight tensor map"); }
         }
     }
@@ -668,6 +669,14 @@ vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* w_packe
     cudaError_t e;
     if (tc) {
         ConvTcPlan plan{};
+        if (a.residual && a.residual != (const float*)a.y) {
+            // the tensor-core kernel accumulates into its output: seed it with the residual
+            const size_t n = (size_t)a.B * a.H * a.W * a.Cout * sizeof(float);
+            e = a.out_dtype == VD_F32 ? cudaMemcpyAsync(a.y, a.residual, n, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream)
+                                      : cudaErrorInvalidValue;
+            if (e != cudaSuccess) return cuda_fail(nullptr, e, "vd_op_conv2d (a residual needs an fp32 output)");
+            a.residual = (const float*)a.y;
+        }
         e = conv_tc_prepare(a, &plan);
         if (e == cudaSuccess) e = launch_conv_tc(a, plan, nullptr, (cudaStream_t)cuda_stream);
     } else {

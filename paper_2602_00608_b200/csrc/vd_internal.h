@@ -15,7 +15,7 @@ struct ConvArgs {
     const float* bias;      // [Cout] or null
     const float* scale;     // [B,Cin] or null
     const float* shift;     // [B,Cin] or null
-    const float* residual;  // fp32 NHWC [B,H,W,Cout] or null
+    const float* residual;  // fp32 NHWC [B,H,W,Cout] or null; the tensor-core kernel needs residual == y (accumulate in place)
     void* y;                // out_dtype, NHWC [B,H,W,Cout] or NCHW [B,Cout,H,W]
     int B, Hs, Ws;          // source resolution
     int H, W;               // output resolution (= source, or 2x source with upsample)
@@ -84,6 +84,9 @@ cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int 
 struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
     unsigned char tmap2[128];   // weights of the fused shortcut (copy of tmap when unused)
+    unsigned char tmap_y[128];  // output tensor (NHWC outputs leave through bulk tensor stores)
+    void* y;                    // the output address tmap_y was built for
+    int batch;                  // frames covered by tmap_y
     int bn;
     int valid;
 };
