@@ -54,6 +54,8 @@ typedef enum { VD_ARCH_TINY = 0, VD_ARCH_SDVAE = 1 } vd_arch;
 
 /* vd_config.flags */
 #define VD_FLAG_FORCE_SIMT 0x1u   /* run every layer on the plain FFMA kernels (cross-check path) */
+#define VD_FLAG_FUSE_GN_STATS 0x2u /* GroupNorm statistics in the producing convolution's epilogue (a frame's
+                                     result then depends, in the last bits, on the batch it is decoded in) */
 
 typedef struct {
     uint32_t struct_size;       /* sizeof(vd_config), for versioning */
@@ -151,6 +153,8 @@ typedef struct {
     double weight_bytes;        /* parameter bytes read once per launch (shared by the batch) */
     int32_t c_in2;              /* > 0: a 1x1 shortcut on a second input of c_in2 channels is fused in */
     int32_t has_residual;       /* 1: an fp32 residual tensor is added in the epilogue */
+    int32_t fused_gn_channels;  /* > 0: the epilogue also produces the GroupNorm statistics of its output */
+    int32_t reserved;
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);
@@ -161,6 +165,12 @@ VD_API vd_status vd_get_step(vd_handle h, int32_t index, vd_step_info* info);
  * a measurement call, not for the serving path. */
 VD_API vd_status vd_profile(vd_handle h, const void* latents, void* frames, int32_t batch, void* cuda_stream,
                             float* ms, int32_t n_steps);
+
+/* Debug: when `device_buffer` is non-NULL (160*4*2048*8 bytes, zeroed by the caller), every
+ * tensor-core convolution launched afterwards records per-CTA role timelines into it (records
+ * are code << 48 | SM clock; roles: 0 operand producer, 1 MMA issue, 2 epilogue); NULL turns
+ * tracing off.  For kernel timing studies only. */
+VD_API vd_status vd_debug_conv_trace(void* device_buffer, size_t bytes);
 
 /* Debug: makes vd_decode stop after step `index` (so that step's output can be read from the
  * workspace at out_offset); -1 restores the full decode. */

@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <map>
 #include <string>
 #include <vector>
 
@@ -95,10 +96,34 @@ class Planner {
     }
 
     void add_gn(const std::string& name, size_t x_off, int dtype, int H, int W, int C, const std::string& wname) {
-        Step s{};
-        s.kind = VD_STEP_GN_STATS;
         size_t g_off, b_off;
         norm_weight(wname, C, g_off, b_off);
+        // scale/shift buffers alternate, so a convolution can read one set in its prologue while
+        // its epilogue writes the next normalisation's set
+        gn_toggle_ ^= 1;
+        scale_off_ = scale_buf_[gn_toggle_];
+        shift_off_ = shift_buf_[gn_toggle_];
+        // If the tensor was written by a tensor-core convolution, that kernel's epilogue computes
+        // the statistics while the values are still on chip: no separate pass over the tensor.
+        auto it = producer_.find(x_off);
+        const int cpg = C / cfg_.norm_groups;
+        if ((cfg_.flags & VD_FLAG_FUSE_GN_STATS) && it != producer_.end() && cfg_.norm_groups <= kConvStatMaxGroups && (cpg == 4 || cpg == 8 || cpg == 16)) {
+            Step& ps = h_->steps[it->second];
+            if (ps.kind == VD_STEP_CONV && ps.use_tc && !ps.conv.out_nchw && ps.conv.Cout == C && !ps.conv.stat_partial) {
+                ps.conv.stat_partial = ptr<float>(stat_partial_off_);
+                ps.conv.stat_counter = ptr<unsigned int>(h_->status_off + 64);
+                ps.conv.stat_gamma = ptr<float>(g_off);
+                ps.conv.stat_beta = ptr<float>(b_off);
+                ps.conv.stat_scale = ptr<float>(scale_off_);
+                ps.conv.stat_shift = ptr<float>(shift_off_);
+                ps.conv.stat_groups = cfg_.norm_groups;
+                ps.conv.stat_eps = cfg_.norm_eps;
+                ps.info.fused_gn_channels = C;
+                return;
+            }
+        }
+        Step s{};
+        s.kind = VD_STEP_GN_STATS;
         s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
                       ptr<float>(b_off), ptr<float>(scale_off_), ptr<float>(shift_off_), ptr<float>(partial_off_)};
         fill_info(s, name, 0, C, C, 0, 0, H, W, C, VD_F32, 0, -1);
@@ -153,6 +178,7 @@ class Planner {
             s.info.bytes_per_frame += P * Cin2 * 4.0;
             s.info.weight_bytes += (double)Cin2 * Cout * elt(cfg_.dtype);
         }
+        if (!y_is_frames) producer_[y_off] = (int)h_->steps.size();
         h_->steps.push_back(s);
     }
 
@@ -252,8 +278,13 @@ class Planner {
         }
         const int ae = elt(act_dtype());
         h_->status_off = alloc(256);
-        scale_off_ = alloc((size_t)B * max_c * 4);
-        shift_off_ = alloc((size_t)B * max_c * 4);
+        for (int i = 0; i < 2; ++i) {
+            scale_buf_[i] = alloc((size_t)B * max_c * 4);
+            shift_buf_[i] = alloc((size_t)B * max_c * 4);
+        }
+        scale_off_ = scale_buf_[0];
+        shift_off_ = shift_buf_[0];
+        stat_partial_off_ = alloc((size_t)B * 2 * kConvStatMaxGroups * kConvStatMaxCtas * 4);
         partial_off_ = alloc(vd_gn_scratch_bytes(B, cfg_.norm_groups));
         zbuf_ = alloc((size_t)B * P0 * lc * 4);
         xs_[0] = alloc((size_t)B * max_x * 4);
@@ -329,6 +360,9 @@ class Planner {
     size_t cur_ = 0;
     size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
+    size_t scale_buf_[2] = {0, 0}, shift_buf_[2] = {0, 0}, stat_partial_off_ = 0;
+    int gn_toggle_ = 0;
+    std::map<size_t, int> producer_;     // workspace offset of a tensor -> step that wrote it last
     int cur_x_ = 0;
 };
 
@@ -346,7 +380,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~VD_FLAG_FORCE_SIMT) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_FUSE_GN_STATS)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -435,6 +469,7 @@ vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, floa
 }  // namespace
 
 namespace vd {
+extern unsigned long long* g_conv_trace;
 void set_last_error(const char* msg) { g_last_error = msg ? msg : ""; }
 }  // namespace vd
 
@@ -588,6 +623,13 @@ vd_status vd_profile(vd_handle h, const void* latents, void* frames, int32_t bat
                      int32_t n_steps) {
     if (!ms) return fail(h, VD_ERR_INVALID_ARG, "ms is NULL");
     return decode_impl(h, latents, nullptr, 0.f, nullptr, nullptr, frames, batch, cuda_stream, ms, n_steps);
+}
+
+vd_status vd_debug_conv_trace(void* device_buffer, size_t bytes) {
+    if (device_buffer && bytes < (size_t)kConvStatMaxCtas * 4 * kConvTraceEvents * sizeof(unsigned long long))
+        return fail(nullptr, VD_ERR_INVALID_ARG, "trace buffer too small");
+    vd::g_conv_trace = (unsigned long long*)device_buffer;
+    return VD_OK;
 }
 
 vd_status vd_debug_stop_after(vd_handle h, int32_t index) {

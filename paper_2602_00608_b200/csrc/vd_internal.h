@@ -26,7 +26,21 @@ struct ConvArgs {
     const void* w2;         // packed bf16 [Cout][Cin2]
     const float* bias2;     // [Cout] or null
     int Cin2;
+    // optional fused GroupNorm statistics of the output (tensor-core kernel only): per-(frame,
+    // channel) scale/shift for the normalisation that consumes y
+    float* stat_partial;        // scratch: [B][2][64][grid] per-CTA sums and sums of squares
+    unsigned int* stat_counter; // zero before the launch; the kernel leaves it zero
+    const float* stat_gamma;    // [Cout]
+    const float* stat_beta;     // [Cout]
+    float* stat_scale;          // [B,Cout] out
+    float* stat_shift;          // [B,Cout] out
+    int stat_groups;
+    float stat_eps;
+    unsigned long long* trace;  // debug: per-CTA role timelines (null in production)
 };
+constexpr int kConvTraceEvents = 2048;    // per (CTA, role)
+constexpr int kConvStatMaxGroups = 64;
+constexpr int kConvStatMaxCtas = 160;
 
 struct GnArgs {
     const void* x;          // NHWC [B,H,W,C]

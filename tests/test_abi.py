@@ -37,14 +37,14 @@ def test_struct_sizes_match_the_header_layout(vd):
     assert ctypes.sizeof(vd.VdConfig) == 44
     assert ctypes.sizeof(vd.VdTensor) == 56
     assert ctypes.sizeof(vd.VdConvDesc) == 56
-    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 8
+    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 16
 
 
 def test_query_workspace_is_host_only_and_scales_with_batch(vd):
     c1 = vd.make_config("sdvae", "bf16", 60, 90, 1, 32, 1e-6)
     c8 = vd.make_config("sdvae", "bf16", 60, 90, 8, 32, 1e-6)
     b1, b8 = vd.query_workspace(c1), vd.query_workspace(c8)
-    assert 1.0e9 < b1 < 2.5e9          # two fp32 stream buffers of 345600 x 256 dominate
+    assert 0.8e9 < b1 < 2.5e9          # two fp32 stream buffers of 345600 x 256 dominate
     assert 6 * b1 < b8 < 8.01 * b1
     t = vd.query_workspace(vd.make_config("tiny", "f32", 8, 8, 1, 8, 1e-6))
     assert t < 8e6
