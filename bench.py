@@ -64,13 +64,6 @@ def contract_roofline_us(steps, peaks, batch, stream_bytes=2):
             else:
                 by = 4 * P * s["c_in"] * stream_bytes
         wb = s["weight_bytes"]
-        if s.get("fused_gn_channels", 0) > 0:
-            # GroupNorm statistics produced in this layer's epilogue: the contract counts the
-            # statistics pass as a layer of its own (one read of the tensor)
-            gb = s["out_h"] * s["out_w"] * s["fused_gn_channels"] * (stream_bytes if stream_bytes is not None else
-                                                                  (2 if s["out_dtype"] == 1 else 4))
-            total += gb / bw
-            byts += gb
         if s.get("c_in2", 0) > 0 and stream_bytes is not None:
             # a fused 1x1 shortcut: the contract counts it as a layer of its own (in, out, weights once)
             P = s["out_h"] * s["out_w"]

@@ -54,8 +54,6 @@ typedef enum { VD_ARCH_TINY = 0, VD_ARCH_SDVAE = 1 } vd_arch;
 
 /* vd_config.flags */
 #define VD_FLAG_FORCE_SIMT 0x1u   /* run every layer on the plain FFMA kernels (cross-check path) */
-#define VD_FLAG_FUSE_GN_STATS 0x2u /* GroupNorm statistics in the producing convolution's epilogue (a frame's
-                                     result then depends, in the last bits, on the batch it is decoded in) */
 
 typedef struct {
     uint32_t struct_size;       /* sizeof(vd_config), for versioning */
@@ -153,8 +151,7 @@ typedef struct {
     double weight_bytes;        /* parameter bytes read once per launch (shared by the batch) */
     int32_t c_in2;              /* > 0: a 1x1 shortcut on a second input of c_in2 channels is fused in */
     int32_t has_residual;       /* 1: an fp32 residual tensor is added in the epilogue */
-    int32_t fused_gn_channels;  /* > 0: the epilogue also produces the GroupNorm statistics of its output */
-    int32_t reserved;
+    int32_t reserved[2];
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);

@@ -15,7 +15,6 @@ VD_OK, VD_ERR_INVALID_ARG, VD_ERR_UNSUPPORTED, VD_ERR_WORKSPACE, VD_ERR_CUDA, VD
 VD_F32, VD_BF16 = 0, 1
 VD_ARCH_TINY, VD_ARCH_SDVAE = 0, 1
 VD_FLAG_FORCE_SIMT = 0x1
-VD_FLAG_FUSE_GN_STATS = 0x2
 VD_IMPL_AUTO, VD_IMPL_SIMT, VD_IMPL_TC = 0, 1, 2
 VD_STEP_INGEST, VD_STEP_GN_STATS, VD_STEP_CONV, VD_STEP_ATTENTION = 0, 1, 2, 3
 STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", -3: "VD_ERR_WORKSPACE",
@@ -45,7 +44,7 @@ class VdStepInfo(Structure):
                 ("out_h", c_int32), ("out_w", c_int32), ("out_channels", c_int32), ("out_dtype", c_int32),
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
                 ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
-                ("has_residual", c_int32), ("fused_gn_channels", c_int32), ("reserved", c_int32)]
+                ("has_residual", c_int32), ("reserved", c_int32 * 2)]
 
 
 class VdConvDesc(Structure):

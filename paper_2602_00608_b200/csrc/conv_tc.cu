@@ -33,6 +33,7 @@
 
 #include <algorithm>
 
+#include "conv_tile.cuh"
 #include "tc_common.cuh"
 #include "vd_internal.h"
 
@@ -41,22 +42,9 @@ namespace vd {
 namespace {
 
 using namespace tc;
+using namespace convtile;
 
-constexpr int TILE_H = 16, TILE_W = 8;                               // one MMA tile: 128 output pixels
-constexpr int PH = TILE_H + 2, PW = TILE_W + 2, NPIX = PH * PW;     // 18 x 10 = 180 halo pixels
-constexpr int A_TILE_BYTES = (NPIX * 128 + 1023) / 1024 * 1024;      // one 64-channel chunk of one halo tile: 180 rows of 128 B
-constexpr int ITEMS = NPIX * 8;                                      // (pixel, 8-channel group) pairs per tile chunk
-constexpr int NUM_PRODUCER_WARPS = 15;
-constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // 480 = ITEMS / 3: three pairs per thread
-constexpr int BATCH = ITEMS / NUM_PRODUCERS;                         // 3
-static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the halo chunk exactly");
-constexpr int TMA_WARP = 15;
-constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
-constexpr int MMA_WARP = 20;
-constexpr int NUM_THREADS = 21 * 32;
 constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
-constexpr int STAT_MAX_GROUPS = 64;                                  // GroupNorm groups the fused statistics can hold
-constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixels x 128 B: one output slice in smem
 
 // BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
 // item is two 16x8-pixel tiles whose MMAs consume every weight stage together, which halves the
@@ -64,114 +52,26 @@ constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixe
 template <int BN> struct TileCfg {
     static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item
     static constexpr int B_STAGE_BYTES = BN * 128;                   // BN rows x 64 bf16
-    static constexpr int B_STAGES = BN == 256 ? 4 : (BN == 128 ? 5 : 8);
+    static constexpr int B_STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int B_GROUP = 2;                                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
-    static constexpr int SMEM_OUT = BN >= 128 ? 3 * OUT_SLICE_BYTES : 0;   // rotating output / residual slices
+    static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
-    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + 512 + 2048 + 1024;  // + barriers + statistics + alignment slack
+    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + 512 + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
     static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
 };
-
-struct Raw8 { uint4 lo, hi; };   // eight channels of one pixel: bf16 -> lo only; fp32 -> lo + hi
-
-// bf16: the thread's 16 bytes are channels [8j, 8j+8) of the chunk.  fp32: two 16-byte loads,
-// channels [4j, 4j+4) and [32+4j, 32+4j+4), so that the eight threads of a pixel read two
-// contiguous 128-byte lines.
-__device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix_off, int c0, int j, Raw8& r) {
-    if (is_bf16) {
-        r.lo = __ldg((const uint4*)((const __nv_bfloat16*)x + pix_off + c0 + j * 8));
-    } else {
-        const float* p = (const float*)x + pix_off + c0 + j * 4;
-        const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 32));
-        r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
-        r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
-    }
-}
-__device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[8]) {
-    if (is_bf16) {
-        const uint32_t w[4] = {r.lo.x, r.lo.y, r.lo.z, r.lo.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[2 * i] = __uint_as_float(w[i] << 16);
-            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    } else {
-        v[0] = __uint_as_float(r.lo.x); v[1] = __uint_as_float(r.lo.y); v[2] = __uint_as_float(r.lo.z); v[3] = __uint_as_float(r.lo.w);
-        v[4] = __uint_as_float(r.hi.x); v[5] = __uint_as_float(r.hi.y); v[6] = __uint_as_float(r.hi.z); v[7] = __uint_as_float(r.hi.w);
-    }
-}
-
-// Per-group sum and sum of squares of 32 consecutive channels (registers v[32]) of the 32 pixels
-// a warp holds, added to the warp's accumulators in shared memory ([2][STAT_MAX_GROUPS]: sums,
-// then sums of squares).  The 2*32/CPG lane-local values are reduced across the warp with a
-// halving butterfly (a fixed order, so the result is reproducible).
-template <int CPG>
-__device__ __forceinline__ void warp_group_stats(const float (&v)[32], bool inside, int lane, float* wacc, int g0) {
-    constexpr int NG = 32 / CPG, NV = 2 * NG;
-    float vals[NV];
-#pragma unroll
-    for (int g = 0; g < NG; ++g) {
-        float s = 0.f, q = 0.f;
-#pragma unroll
-        for (int e = 0; e < CPG; ++e) {
-            const float x = v[g * CPG + e];
-            s += x;
-            q = fmaf(x, x, q);
-        }
-        vals[g] = inside ? s : 0.f;
-        vals[NG + g] = inside ? q : 0.f;
-    }
-    // after the step with lane mask M a lane keeps the half of the values selected by its bit M
-    int idx = 0;
-#pragma unroll
-    for (int half = NV / 2, mask = 16; half >= 1; half >>= 1, mask >>= 1) {
-        const bool upper = (lane & mask) != 0;
-#pragma unroll
-        for (int i = 0; i < half; ++i) {
-            const float send = upper ? vals[i] : vals[i + half];
-            const float keep = upper ? vals[i + half] : vals[i];
-            vals[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
-        }
-        idx += upper ? half : 0;
-    }
-    // NV values took log2(NV) steps; the remaining lane bits still hold partial sums of the same value
-    constexpr int STEPS = NV == 16 ? 4 : (NV == 8 ? 3 : 2);
-#pragma unroll
-    for (int mask = 16 >> STEPS; mask >= 1; mask >>= 1) vals[0] += __shfl_xor_sync(0xffffffffu, vals[0], mask);
-    if ((lane & ((32 >> STEPS) - 1)) == 0) {
-        const int stat = idx / NG, g = idx - stat * NG;
-        wacc[stat * STAT_MAX_GROUPS + g0 + g] += vals[0];
-    }
-}
 
 struct Bars {                    // lives in shared memory
     uint64_t a_full[MAX_A_STAGES], a_empty[MAX_A_STAGES];
     uint64_t b_full[MAX_B_STAGES], b_empty[MAX_B_STAGES];
     uint64_t acc_full[2], acc_empty[2];
     uint64_t epi_sync;           // rendezvous of the 128 epilogue threads (a bounded stand-in for bar.sync)
-    uint64_t res_full[3];        // residual slice has landed in output buffer i
     uint32_t tmem_base;
     uint32_t abort_flag;
-    uint32_t is_last;
-};
-
-struct Tile { int tx0, ty0, n0, b; };
-
-// Debug timeline: role r of this CTA appends (code << 48 | clock) records when a trace buffer is given.
-struct Tracer {
-    unsigned long long* p;
-    int n;
-    __device__ __forceinline__ void init(unsigned long long* base, int role) {
-        p = base ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
-        n = 0;
-    }
-    __device__ __forceinline__ void mark(unsigned code) {
-        if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFull);
-    }
 };
 
 // Tiles are numbered (frame, channel block, tile row, tile column), column fastest.  Every CTA
@@ -232,7 +132,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
         mbar_init(smem_u32(&bars->epi_sync), 128);
-        for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&bars->res_full[i]), 1);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -349,59 +248,20 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         // ------------------------------------------------ epilogue
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
         const int m = ew * 32 + lane;                        // accumulator row = pixel of the MMA tile
-        const int et = tid - EPI_WARP0 * 32;                 // 0..127
-        const bool leader = et == 0;                         // issues the bulk loads / stores
-        const bool want_stats = OUT_MODE != 2 && a.stat_partial != nullptr;
-        // y holds the residual stream.  Plain case: the tile is added into it by a bulk reduce-add (the
-        // residual never enters the SM).  With fused statistics the final values are needed on chip,
-        // so the residual slice is loaded, added and the sum stored back.
-        const bool has_res = a.residual != nullptr && want_stats;
-        const bool reduce_add = a.residual != nullptr && !want_stats;
-        const int cpg = want_stats ? a.Cout / a.stat_groups : 4;
-        float* stat_acc = (float*)(smem + Cfg::SMEM_B + Cfg::SMEM_OUT + Cfg::SMEM_A + sizeof(Bars));   // [4 warps][2][64]
+        const bool leader = tid == EPI_WARP0 * 32;           // issues the bulk stores
+        const bool reduce_add = a.residual != nullptr;       // y is the residual stream: the tile is added into it
         Tracer tr; tr.init(leader ? a.trace : nullptr, 2);
         bool ok = true;
         int n_item = 0;
         uint32_t n_slice = 0, sync_phase = 0;
-        int stat_b = -1;                                     // frame the shared-memory statistics belong to
         auto epi_rendezvous = [&]() {                        // all 128 epilogue threads meet here; bounded like every wait
             mbar_arrive(smem_u32(&bars->epi_sync));
             const bool r = mbar_wait(smem_u32(&bars->epi_sync), sync_phase, abort_flag);
             sync_phase ^= 1;
             return r;
         };
-        // moves this CTA's statistics of frame `b` to global memory (one record per CTA and frame)
-        auto flush_stats = [&](int b) {
-            bool r = epi_rendezvous();
-            if (et < 2 * STAT_MAX_GROUPS) {
-                float tot = 0.f;
-#pragma unroll
-                for (int w4 = 0; w4 < 4; ++w4) tot += stat_acc[w4 * 2 * STAT_MAX_GROUPS + et];
-                // layout [frame][stat][group][cta]: a warp of the finalising CTA reads 32 CTAs' records at once
-                a.stat_partial[(((size_t)b * 2 * STAT_MAX_GROUPS) + et) * gridDim.x + blockIdx.x] = tot;
-            }
-            r = epi_rendezvous() && r;
-            for (int i = et; i < 4 * 2 * STAT_MAX_GROUPS; i += 128) stat_acc[i] = 0.f;
-            return epi_rendezvous() && r;
-        };
-        if (want_stats) {
-            for (int i = et; i < 4 * 2 * STAT_MAX_GROUPS; i += 128) stat_acc[i] = 0.f;
-            ok = __all_sync(0xffffffffu, epi_rendezvous());
-        }
         constexpr int CS = OUT_MODE == 1 ? 64 : 32;          // channels per 128-byte output slice
         constexpr int NS = BN >= CS ? BN / CS : 1;
-        // coordinates of the slice after (t, cnt, slot, sidx), for the residual prefetch
-        auto next_slice = [&](int t, int cnt, int slot, int sidx, Tile& tl, int& ns) {
-            if (sidx + 1 < NS) { tl = sched.get(t + slot, BN); ns = sidx + 1; return true; }
-            if (slot + 1 < cnt) { tl = sched.get(t + slot + 1, BN); ns = 0; return true; }
-            if (t + cnt < sched.end) { tl = sched.get(t + cnt, BN); ns = 0; return true; }
-            return false;
-        };
-        if (OUT_MODE != 2 && has_res && leader && sched.begin < sched.end) {
-            const Tile tl = sched.get(sched.begin, BN);     // first residual slice
-            mbar_arrive_expect_tx(smem_u32(&bars->res_full[0]), OUT_SLICE_BYTES);
-            tma_load_4d(smem_u32(smem_out), &tmap_y, tl.n0, tl.tx0, tl.ty0, tl.b, smem_u32(&bars->res_full[0]));
-        }
         for (int t = sched.begin; t < sched.end && ok; ++n_item) {
             const int cnt = sched.count(t);
             const int buf = n_item % NBUF;
@@ -416,9 +276,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const Tile tl = sched.get(t + slot, BN);
                 const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
                 const bool last_tile = slot == cnt - 1;
-                const int oy = tl.ty0 + (m >> 3), ox = tl.tx0 + (m & 7);
-                const bool inside = oy < a.H && ox < a.W;
                 if (OUT_MODE == 2) {
+                    const int oy = tl.ty0 + (m >> 3), ox = tl.tx0 + (m & 7);
                     uint32_t r[16];
                     tmem_ld16(tacc, r);
                     tmem_ld_wait();
@@ -427,7 +286,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
                     }
-                    if (inside) {
+                    if (oy < a.H && ox < a.W) {
 #pragma unroll
                         for (int co = 0; co < 16; ++co) {
                             if (co < a.Cout) {
@@ -439,38 +298,16 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         }
                     }
                 } else {
-                    if (want_stats && tl.b != stat_b) {
-                        if (stat_b >= 0) ok = __all_sync(0xffffffffu, flush_stats(stat_b));
-                        stat_b = tl.b;
-                        if (!ok) break;
-                    }
                     // The tile leaves through shared memory in 128-byte-wide slices (32 fp32 or 64
                     // bf16 channels), written row-per-thread in the 128B-swizzled layout of a bulk
-                    // tensor copy; the copy clips the ragged image edge by itself.  Three slice
-                    // buffers rotate: one being stored, one being filled, one receiving the next
-                    // slice of the residual stream.
+                    // tensor store; the store clips the ragged image edge by itself.
 #pragma unroll 1
                     for (int sidx = 0; sidx < NS; ++sidx, ++n_slice) {
-                        uint8_t* obuf = smem_out + (n_slice % 3) * OUT_SLICE_BYTES;
+                        uint8_t* obuf = smem_out + (n_slice & 1) * OUT_SLICE_BYTES;
                         tr.mark(12);
-                        if (leader) {
-                            bulk_wait_group_read<1>();                // the store issued two slices ago has drained its buffer
-                            Tile ntl;
-                            int nsidx;
-                            if (has_res && next_slice(t, cnt, slot, sidx, ntl, nsidx)) {
-                                const uint32_t nb = (n_slice + 1) % 3;
-                                mbar_arrive_expect_tx(smem_u32(&bars->res_full[nb]), OUT_SLICE_BYTES);
-                                tma_load_4d(smem_u32(smem_out + nb * OUT_SLICE_BYTES), &tmap_y, ntl.n0 + nsidx * CS, ntl.tx0, ntl.ty0,
-                                            ntl.b, smem_u32(&bars->res_full[nb]));
-                            }
-                        }
+                        if (leader) bulk_wait_group_read<1>();        // the store that last read this buffer is done
                         ok = __all_sync(0xffffffffu, epi_rendezvous());
                         if (!ok) break;
-                        if (has_res) {
-                            ok = mbar_wait(smem_u32(&bars->res_full[n_slice % 3]), (n_slice / 3) & 1, abort_flag);
-                            ok = __all_sync(0xffffffffu, ok);
-                            if (!ok) break;
-                        }
                         tr.mark(13);
                         uint8_t* orow = obuf + m * 128;
 #pragma unroll
@@ -502,38 +339,15 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 }
                             }
                             if (OUT_MODE == 0) {
-                                if (has_res) {
-#pragma unroll
-                                    for (int c = 0; c < 8; ++c) {
-                                        const float4 x = *(const float4*)(orow + ((c ^ (m & 7)) << 4));
-                                        v[4 * c] += x.x; v[4 * c + 1] += x.y; v[4 * c + 2] += x.z; v[4 * c + 3] += x.w;
-                                    }
-                                }
 #pragma unroll
                                 for (int c = 0; c < 8; ++c)
                                     *(float4*)(orow + ((c ^ (m & 7)) << 4)) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
                             } else {
 #pragma unroll
-                                for (int c = 0; c < 4; ++c) {
-                                    const uint4 pk = make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
-                                                                pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
-                                    *(uint4*)(orow + (((h * 4 + c) ^ (m & 7)) << 4)) = pk;
-                                    if (want_stats) {         // statistics are those of the values as stored
-                                        const uint32_t w4[4] = {pk.x, pk.y, pk.z, pk.w};
-#pragma unroll
-                                        for (int e = 0; e < 4; ++e) {
-                                            v[8 * c + 2 * e] = __uint_as_float(w4[e] << 16);
-                                            v[8 * c + 2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
-                                        }
-                                    }
-                                }
-                            }
-                            if (want_stats) {
-                                float* wacc = stat_acc + ew * 2 * STAT_MAX_GROUPS;
-                                const int g0 = co / cpg;          // first group of these 32 channels
-                                if (cpg == 4) warp_group_stats<4>(v, inside, lane, wacc, g0);
-                                else if (cpg == 8) warp_group_stats<8>(v, inside, lane, wacc, g0);
-                                else warp_group_stats<16>(v, inside, lane, wacc, g0);
+                                for (int c = 0; c < 4; ++c)
+                                    *(uint4*)(orow + (((h * 4 + c) ^ (m & 7)) << 4)) =
+                                        make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
+                                                   pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
                             }
                         }
                         tr.mark(14);
@@ -552,52 +366,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             t += cnt;
         }
         if (leader) bulk_wait_group<0>();                    // all stores have landed before the CTA retires
-        if (want_stats && ok) {
-            if (stat_b >= 0) ok = __all_sync(0xffffffffu, flush_stats(stat_b));
-            // The CTA that finishes last turns the per-CTA records into the next layer's per-(frame,
-            // channel) scale and shift: scale = gamma * rstd, shift = beta - mean * scale.
-            if (ok) {
-                if (leader) {
-                    __threadfence();
-                    const unsigned int prev = atomicAdd(a.stat_counter, 1u);
-                    bars->is_last = (prev == gridDim.x - 1) ? 1u : 0u;
-                }
-                ok = __all_sync(0xffffffffu, epi_rendezvous());
-            }
-            if (ok && bars->is_last) {
-                __threadfence();
-                const int G = a.stat_groups;
-                const int tiles_per_frame = sched.tiles * sched.nblk;
-                const double count = (double)a.H * a.W * cpg;
-                for (int row = ew; row < a.B * G; row += 4) {       // one (frame, group) per warp at a time
-                    const int b = row / G, g = row - b * G;
-                    // CTAs whose tile range meets this frame wrote a record; sum them in a fixed order
-                    double s = 0.0, q = 0.0;
-                    for (int c = lane; c < (int)gridDim.x; c += 32) {
-                        const long long cb = ((long long)sched.total * c) / gridDim.x, ce = ((long long)sched.total * (c + 1)) / gridDim.x;
-                        if (ce > (long long)b * tiles_per_frame && cb < (long long)(b + 1) * tiles_per_frame) {
-                            s += (double)__ldcg(a.stat_partial + (((size_t)b * 2 * STAT_MAX_GROUPS) + g) * gridDim.x + c);
-                            q += (double)__ldcg(a.stat_partial + (((size_t)b * 2 * STAT_MAX_GROUPS) + STAT_MAX_GROUPS + g) * gridDim.x + c);
-                        }
-                    }
-#pragma unroll
-                    for (int d = 16; d > 0; d >>= 1) {
-                        s += __shfl_xor_sync(0xffffffffu, s, d);
-                        q += __shfl_xor_sync(0xffffffffu, q, d);
-                    }
-                    const double mean = s / count;
-                    const double var = fmax(q / count - mean * mean, 0.0);
-                    const float rstd = (float)(1.0 / sqrt(var + (double)a.stat_eps));
-                    for (int cc = lane; cc < cpg; cc += 32) {
-                        const int ch = g * cpg + cc;
-                        const float sc = a.stat_gamma[ch] * rstd;
-                        a.stat_scale[(size_t)b * a.Cout + ch] = sc;
-                        a.stat_shift[(size_t)b * a.Cout + ch] = a.stat_beta[ch] - (float)mean * sc;
-                    }
-                }
-                if (leader) *a.stat_counter = 0u;            // ready for the next launch
-            }
-        }
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
         if (lane == 0) {
@@ -611,10 +379,12 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
                     for (int tap = 0; tap < ntap; ++tap) {
-                        tr.mark(30);
-                        ok = mbar_wait(smem_u32(&bars->b_empty[stage]), phase ^ 1, abort_flag);
-                        if (!ok) break;
-                        tr.mark(31);
+                        if (stage % Cfg::B_GROUP == 0) {     // stages come back in groups (see the MMA thread)
+                            tr.mark(30);
+                            ok = mbar_wait(smem_u32(&bars->b_empty[stage / Cfg::B_GROUP]), phase ^ 1, abort_flag);
+                            if (!ok) break;
+                            tr.mark(31);
+                        }
                         const uint32_t full = smem_u32(&bars->b_full[stage]);
                         mbar_arrive_expect_tx(full, Cfg::B_STAGE_BYTES);
                         if (second) tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap2, (kc - kchunks) * 64, tl.n0, full);
@@ -675,7 +445,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const int ky = centre ? 1 : tap / 3, kx = centre ? 1 : tap - 3 * (tap / 3);
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
                         uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (uint32_t)(ky * PW + kx) * 8;
-                        uint32_t acc = (kc | tap) != 0;
+                        const uint32_t acc = (kc | tap) != 0;
                         uint32_t td = tmem_d;
                         for (int slot = 0; slot < cnt; ++slot) {
                             umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
@@ -685,7 +455,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             a_lo += A_TILE_BYTES >> 4;
                             td += Cfg::ACC_COLS;
                         }
-                        umma_commit(smem_u32(&bars->b_empty[bs]));
+                        // tcgen05.commit is served at a limited rate (about one per 700 cycles), so weight
+                        // stages are handed back B_GROUP at a time
+                        if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
                         if (++bs == Cfg::B_STAGES) { bs = 0; bph ^= 1; }
                     }
                     umma_commit(smem_u32(&bars->a_empty[as]));
@@ -775,7 +547,7 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     }
     const int tiles = ((a.W + TILE_W - 1) / TILE_W) * ((a.H + TILE_H - 1) / TILE_H);
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
-    int grid = (int)std::min<long long>(total, std::min(num_sms(), kConvStatMaxCtas));
+    int grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
     if (getenv("VD_CONV_GRID")) grid = std::min(grid, atoi(getenv("VD_CONV_GRID")));   // timing studies
     kern<<<grid, NUM_THREADS, TileCfg<BN>::SMEM_TOTAL, s>>>(a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
                                                             *(const CUtensorMap*)plan.tmap_y, status);
@@ -821,6 +593,14 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     } else {
         memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
     }
+    if (bn >= 128) {      // half-height boxes for the two-CTA kernel
+        if (!encode_weights((CUtensorMap*)plan->tmap_half, a.w, a.Cin, taps * padded_cout(a.Cout), bn / 2)) return cudaErrorInvalidValue;
+        if (a.x2) {
+            if (!encode_weights((CUtensorMap*)plan->tmap2_half, a.w2, a.Cin2, a.Cout, bn / 2)) return cudaErrorInvalidValue;
+        } else {
+            memcpy(plan->tmap2_half, plan->tmap_half, sizeof(plan->tmap_half));
+        }
+    }
     if (!a.out_nchw) {
         // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one 128-byte-wide slice of a tile
         EncodeTiledFn enc = get_encode_fn();
@@ -853,6 +633,12 @@ cudaError_t launch_conv_tc(const ConvArgs& a_in, const ConvTcPlan& plan, unsigne
     a.trace = g_conv_trace;
     if (!a.out_nchw && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
+    static const bool one_cta = getenv("VD_CONV_ONE_CTA") != nullptr;                        // timing studies
+    if (!one_cta && plan.bn >= 128 && conv_tc2_supported(a)) {
+        const cudaError_t e = launch_conv_tc2(a, plan, status, s);
+        if (e != cudaErrorNotSupported) return e;
+        (void)cudaGetLastError();
+    }
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2>(a, plan, status, s) : launch_one<16, false, 2>(a, plan, status, s);

@@ -1,0 +1,72 @@
+// Pieces shared by the one-CTA and the two-CTA tensor-core convolution kernels: tile geometry,
+// the operand loader of the prologue, and the debug timeline recorder.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "tc_common.cuh"
+#include "vd_internal.h"
+
+namespace vd {
+namespace convtile {
+
+constexpr int TILE_H = 16, TILE_W = 8;                               // one MMA tile: 128 output pixels
+constexpr int PH = TILE_H + 2, PW = TILE_W + 2, NPIX = PH * PW;     // 18 x 10 = 180 halo pixels
+constexpr int A_TILE_BYTES = (NPIX * 128 + 1023) / 1024 * 1024;      // one 64-channel chunk of one halo tile: 180 rows of 128 B
+constexpr int ITEMS = NPIX * 8;                                      // (pixel, 8-channel group) pairs per tile chunk
+constexpr int NUM_PRODUCER_WARPS = 15;
+constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // 480 = ITEMS / 3: three pairs per thread
+constexpr int BATCH = ITEMS / NUM_PRODUCERS;                         // 3
+static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the halo chunk exactly");
+constexpr int TMA_WARP = 15;
+constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
+constexpr int MMA_WARP = 20;
+constexpr int NUM_THREADS = 21 * 32;
+constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixels x 128 B: one output slice in smem
+
+struct Raw8 { uint4 lo, hi; };   // eight channels of one pixel: bf16 -> lo only; fp32 -> lo + hi
+
+// bf16: the thread's 16 bytes are channels [8j, 8j+8) of the chunk.  fp32: two 16-byte loads,
+// channels [4j, 4j+4) and [32+4j, 32+4j+4), so that the eight threads of a pixel read two
+// contiguous 128-byte lines.
+__device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix_off, int c0, int j, Raw8& r) {
+    if (is_bf16) {
+        r.lo = __ldg((const uint4*)((const __nv_bfloat16*)x + pix_off + c0 + j * 8));
+    } else {
+        const float* p = (const float*)x + pix_off + c0 + j * 4;
+        const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 32));
+        r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
+        r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
+    }
+}
+__device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[8]) {
+    if (is_bf16) {
+        const uint32_t w[4] = {r.lo.x, r.lo.y, r.lo.z, r.lo.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    } else {
+        v[0] = __uint_as_float(r.lo.x); v[1] = __uint_as_float(r.lo.y); v[2] = __uint_as_float(r.lo.z); v[3] = __uint_as_float(r.lo.w);
+        v[4] = __uint_as_float(r.hi.x); v[5] = __uint_as_float(r.hi.y); v[6] = __uint_as_float(r.hi.z); v[7] = __uint_as_float(r.hi.w);
+    }
+}
+
+struct Tile { int tx0, ty0, n0, b; };
+
+// Debug timeline: role r of this CTA appends (code << 48 | clock) records when a trace buffer is given.
+struct Tracer {
+    unsigned long long* p;
+    int n;
+    __device__ __forceinline__ void init(unsigned long long* base, int role) {
+        p = base ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
+        n = 0;
+    }
+    __device__ __forceinline__ void mark(unsigned code) {
+        if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFull);
+    }
+};
+
+}  // namespace convtile
+}  // namespace vd

@@ -3,7 +3,6 @@
 #include <stdio.h>
 #include <string.h>
 
-#include <map>
 #include <string>
 #include <vector>
 
@@ -103,25 +102,6 @@ class Planner {
         gn_toggle_ ^= 1;
         scale_off_ = scale_buf_[gn_toggle_];
         shift_off_ = shift_buf_[gn_toggle_];
-        // If the tensor was written by a tensor-core convolution, that kernel's epilogue computes
-        // the statistics while the values are still on chip: no separate pass over the tensor.
-        auto it = producer_.find(x_off);
-        const int cpg = C / cfg_.norm_groups;
-        if ((cfg_.flags & VD_FLAG_FUSE_GN_STATS) && it != producer_.end() && cfg_.norm_groups <= kConvStatMaxGroups && (cpg == 4 || cpg == 8 || cpg == 16)) {
-            Step& ps = h_->steps[it->second];
-            if (ps.kind == VD_STEP_CONV && ps.use_tc && !ps.conv.out_nchw && ps.conv.Cout == C && !ps.conv.stat_partial) {
-                ps.conv.stat_partial = ptr<float>(stat_partial_off_);
-                ps.conv.stat_counter = ptr<unsigned int>(h_->status_off + 64);
-                ps.conv.stat_gamma = ptr<float>(g_off);
-                ps.conv.stat_beta = ptr<float>(b_off);
-                ps.conv.stat_scale = ptr<float>(scale_off_);
-                ps.conv.stat_shift = ptr<float>(shift_off_);
-                ps.conv.stat_groups = cfg_.norm_groups;
-                ps.conv.stat_eps = cfg_.norm_eps;
-                ps.info.fused_gn_channels = C;
-                return;
-            }
-        }
         Step s{};
         s.kind = VD_STEP_GN_STATS;
         s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
@@ -178,7 +158,6 @@ class Planner {
             s.info.bytes_per_frame += P * Cin2 * 4.0;
             s.info.weight_bytes += (double)Cin2 * Cout * elt(cfg_.dtype);
         }
-        if (!y_is_frames) producer_[y_off] = (int)h_->steps.size();
         h_->steps.push_back(s);
     }
 
@@ -284,7 +263,6 @@ class Planner {
         }
         scale_off_ = scale_buf_[0];
         shift_off_ = shift_buf_[0];
-        stat_partial_off_ = alloc((size_t)B * 2 * kConvStatMaxGroups * kConvStatMaxCtas * 4);
         partial_off_ = alloc(vd_gn_scratch_bytes(B, cfg_.norm_groups));
         zbuf_ = alloc((size_t)B * P0 * lc * 4);
         xs_[0] = alloc((size_t)B * max_x * 4);
@@ -360,9 +338,8 @@ class Planner {
     size_t cur_ = 0;
     size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
-    size_t scale_buf_[2] = {0, 0}, shift_buf_[2] = {0, 0}, stat_partial_off_ = 0;
+    size_t scale_buf_[2] = {0, 0}, shift_buf_[2] = {0, 0};
     int gn_toggle_ = 0;
-    std::map<size_t, int> producer_;     // workspace offset of a tensor -> step that wrote it last
     int cur_x_ = 0;
 };
 
@@ -380,7 +357,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_FUSE_GN_STATS)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~VD_FLAG_FORCE_SIMT) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -626,7 +603,7 @@ vd_status vd_profile(vd_handle h, const void* latents, void* frames, int32_t bat
 }
 
 vd_status vd_debug_conv_trace(void* device_buffer, size_t bytes) {
-    if (device_buffer && bytes < (size_t)kConvStatMaxCtas * 4 * kConvTraceEvents * sizeof(unsigned long long))
+    if (device_buffer && bytes < (size_t)kConvMaxCtas * 4 * kConvTraceEvents * sizeof(unsigned long long))
         return fail(nullptr, VD_ERR_INVALID_ARG, "trace buffer too small");
     vd::g_conv_trace = (unsigned long long*)device_buffer;
     return VD_OK;

@@ -26,21 +26,10 @@ struct ConvArgs {
     const void* w2;         // packed bf16 [Cout][Cin2]
     const float* bias2;     // [Cout] or null
     int Cin2;
-    // optional fused GroupNorm statistics of the output (tensor-core kernel only): per-(frame,
-    // channel) scale/shift for the normalisation that consumes y
-    float* stat_partial;        // scratch: [B][2][64][grid] per-CTA sums and sums of squares
-    unsigned int* stat_counter; // zero before the launch; the kernel leaves it zero
-    const float* stat_gamma;    // [Cout]
-    const float* stat_beta;     // [Cout]
-    float* stat_scale;          // [B,Cout] out
-    float* stat_shift;          // [B,Cout] out
-    int stat_groups;
-    float stat_eps;
     unsigned long long* trace;  // debug: per-CTA role timelines (null in production)
 };
 constexpr int kConvTraceEvents = 2048;    // per (CTA, role)
-constexpr int kConvStatMaxGroups = 64;
-constexpr int kConvStatMaxCtas = 160;
+constexpr int kConvMaxCtas = 160;         // upper bound on the persistent grid (sizes the debug trace)
 
 struct GnArgs {
     const void* x;          // NHWC [B,H,W,C]
@@ -99,6 +88,8 @@ struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
     unsigned char tmap2[128];   // weights of the fused shortcut (copy of tmap when unused)
     unsigned char tmap_y[128];  // output tensor (NHWC outputs leave through bulk tensor stores)
+    unsigned char tmap_half[128];   // weights with half-height boxes (two-CTA kernel: each CTA stages BN/2 rows)
+    unsigned char tmap2_half[128];
     void* y;                    // the output address tmap_y was built for
     int batch;                  // frames covered by tmap_y
     int bn;
@@ -106,6 +97,9 @@ struct alignas(64) ConvTcPlan {
 };
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
+// two-CTA (cta_group::2) variant, conv_tc2.cu; launch_conv_tc routes to it where it applies
+bool conv_tc2_supported(const ConvArgs& a);
+cudaError_t launch_conv_tc2(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
 bool attn_tc_supported(const AttnArgs& a);
 size_t attn_tc_scratch_bytes(int B, int T, int C);
 cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
