@@ -45,6 +45,7 @@ using namespace tc;
 using namespace convtile;
 
 constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
+constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epilogue warp's share of an output slice
 
 // BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
 // item is two 16x8-pixel tiles whose MMAs consume every weight stage together, which halves the
@@ -59,7 +60,8 @@ template <int BN> struct TileCfg {
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
-    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + 512 + 1024;  // + barriers + alignment slack
+    static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
+    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + 512 + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
     static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
@@ -69,7 +71,6 @@ struct Bars {                    // lives in shared memory
     uint64_t a_full[MAX_A_STAGES], a_empty[MAX_A_STAGES];
     uint64_t b_full[MAX_B_STAGES], b_empty[MAX_B_STAGES];
     uint64_t acc_full[2], acc_empty[2];
-    uint64_t epi_sync;           // rendezvous of the 128 epilogue threads (a bounded stand-in for bar.sync)
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -109,7 +110,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     uint8_t* smem_b = smem;
     uint8_t* smem_out = smem + Cfg::SMEM_B;
     uint8_t* smem_a = smem_out + Cfg::SMEM_OUT;
-    Bars* bars = (Bars*)(smem_a + Cfg::SMEM_A);
+    uint8_t* smem_bias = smem_a + Cfg::SMEM_A;
+    Bars* bars = (Bars*)(smem_bias + Cfg::SMEM_BIAS);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -131,7 +133,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), 1); }
         for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
-        mbar_init(smem_u32(&bars->epi_sync), 128);
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -246,42 +247,30 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------ epilogue
+        // Each warp owns a quarter of the accumulator rows (32 pixels = four rows of the 16x8 tile)
+        // and works on its own: no synchronisation between the four warps.  TMEM reads are issued
+        // one column block ahead of the one being processed.
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
-        const int m = ew * 32 + lane;                        // accumulator row = pixel of the MMA tile
-        const bool leader = tid == EPI_WARP0 * 32;           // issues the bulk stores
         const bool reduce_add = a.residual != nullptr;       // y is the residual stream: the tile is added into it
-        Tracer tr; tr.init(leader ? a.trace : nullptr, 2);
+        Tracer tr; tr.init(tid == EPI_WARP0 * 32 ? a.trace : nullptr, 2);
         bool ok = true;
         int n_item = 0;
-        uint32_t n_slice = 0, sync_phase = 0;
-        auto epi_rendezvous = [&]() {                        // all 128 epilogue threads meet here; bounded like every wait
-            mbar_arrive(smem_u32(&bars->epi_sync));
-            const bool r = mbar_wait(smem_u32(&bars->epi_sync), sync_phase, abort_flag);
-            sync_phase ^= 1;
-            return r;
-        };
-        constexpr int CS = OUT_MODE == 1 ? 64 : 32;          // channels per 128-byte output slice
-        constexpr int NS = BN >= CS ? BN / CS : 1;
-        for (int t = sched.begin; t < sched.end && ok; ++n_item) {
-            const int cnt = sched.count(t);
-            const int buf = n_item % NBUF;
-            tr.mark(10);
-            ok = mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld below is warp-collective
-            if (!ok) break;
-            tc_fence_after();
-            tr.mark(11);
-#pragma unroll 1
-            for (int slot = 0; slot < cnt && ok; ++slot) {
-                const Tile tl = sched.get(t + slot, BN);
-                const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
-                const bool last_tile = slot == cnt - 1;
-                if (OUT_MODE == 2) {
+        uint32_t n_slice = 0;
+        if (OUT_MODE == 2) {
+            for (int t = sched.begin; t < sched.end && ok; ++n_item) {
+                const int cnt = sched.count(t);
+                const int buf = n_item % NBUF;
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
+                for (int slot = 0; slot < cnt; ++slot) {
+                    const Tile tl = sched.get(t + slot, BN);
+                    const int m = ew * 32 + lane;
                     const int oy = tl.ty0 + (m >> 3), ox = tl.tx0 + (m & 7);
                     uint32_t r[16];
-                    tmem_ld16(tacc, r);
+                    tmem_ld16(tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16), r);
                     tmem_ld_wait();
-                    if (last_tile) {
+                    if (slot == cnt - 1) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
@@ -297,75 +286,97 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             }
                         }
                     }
-                } else {
-                    // The tile leaves through shared memory in 128-byte-wide slices (32 fp32 or 64
-                    // bf16 channels), written row-per-thread in the 128B-swizzled layout of a bulk
-                    // tensor store; the store clips the ragged image edge by itself.
+                }
+                t += cnt;
+            }
+        } else {
+            // The warp's 32 rows leave through shared memory as 128-byte-wide slices (32 fp32 or 64
+            // bf16 channels), written row-per-lane in the 128B-swizzled layout of a bulk tensor
+            // store of a [4 rows x 8 pixels x slice] box; the store clips the ragged image edge.
+            constexpr int NP = BN / 32;                       // 32-column passes per tile
+            constexpr int PPS = OUT_MODE == 1 ? 2 : 1;        // passes per 128-byte slice
+            uint8_t* wout = smem_out + ew * (2 * WARP_SLICE_BYTES);         // this warp's two slice buffers
+            float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
+            int bias_n0 = -1;
+            for (int t = sched.begin; t < sched.end && ok; ++n_item) {
+                const int cnt = sched.count(t);
+                const int buf = n_item % NBUF;
+                tr.mark(10);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
+                if (!ok) break;
+                tc_fence_after();
+                tr.mark(11);
 #pragma unroll 1
-                    for (int sidx = 0; sidx < NS; ++sidx, ++n_slice) {
-                        uint8_t* obuf = smem_out + (n_slice & 1) * OUT_SLICE_BYTES;
-                        tr.mark(12);
-                        if (leader) bulk_wait_group_read<1>();        // the store that last read this buffer is done
-                        ok = __all_sync(0xffffffffu, epi_rendezvous());
-                        if (!ok) break;
-                        tr.mark(13);
-                        uint8_t* orow = obuf + m * 128;
+                for (int slot = 0; slot < cnt; ++slot) {
+                    const Tile tl = sched.get(t + slot, BN);
+                    if (tl.n0 != bias_n0) {                   // (re)load bias (+ shortcut bias) of this channel block
+                        __syncwarp();
+                        for (int i = lane; i < BN; i += 32)
+                            wbias[i] = (a.bias ? __ldg(a.bias + tl.n0 + i) : 0.f) + (a.bias2 ? __ldg(a.bias2 + tl.n0 + i) : 0.f);
+                        bias_n0 = tl.n0;
+                        __syncwarp();
+                    }
+                    const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
+                    const bool last_tile = slot == cnt - 1;
+                    uint32_t ra[32], rb[32];
+                    tmem_ld32(tacc, ra);
+                    tmem_ld_wait();
 #pragma unroll
-                        for (int h = 0; h < CS / 32; ++h) {
-                            uint32_t r[32];
-                            tmem_ld32(tacc + (uint32_t)(sidx * CS + h * 32), r);
-                            tmem_ld_wait();
-                            if (last_tile && sidx == NS - 1 && h == CS / 32 - 1) {   // accumulators fully read
-                                tc_fence_before();
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                    for (int p = 0; p < NP; ++p) {
+                        uint32_t (&rc)[32] = (p & 1) ? rb : ra;          // this pass
+                        uint32_t (&rn)[32] = (p & 1) ? ra : rb;          // next pass, in flight while this one is processed
+                        if (p + 1 < NP) tmem_ld32(tacc + (uint32_t)((p + 1) * 32), rn);
+                        const int sl = p / PPS, h = p % PPS;              // slice, half of the slice
+                        uint8_t* obuf = wout + ((n_slice + sl) & 1) * WARP_SLICE_BYTES;
+                        if (h == 0) {
+                            if (lane == 0) bulk_wait_group_read<1>();     // the store that last read this buffer is done
+                            __syncwarp();
+                        }
+                        uint8_t* orow = obuf + lane * 128;
+                        const float4* bp = (const float4*)(wbias + p * 32);
+                        if (OUT_MODE == 0) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                const float4 tb = bp[c];
+                                *(float4*)(orow + ((c ^ (lane & 7)) << 4)) =
+                                    make_float4(__uint_as_float(rc[4 * c]) + tb.x, __uint_as_float(rc[4 * c + 1]) + tb.y,
+                                                __uint_as_float(rc[4 * c + 2]) + tb.z, __uint_as_float(rc[4 * c + 3]) + tb.w);
                             }
-                            const int co = tl.n0 + sidx * CS + h * 32;
-                            float v[32];
+                        } else {
 #pragma unroll
-                            for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
-                            if (a.bias) {
-#pragma unroll
-                                for (int q = 0; q < 32; q += 4) {
-                                    const float4 tb = __ldg((const float4*)(a.bias + co + q));
-                                    v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
-                                }
-                            }
-                            if (a.bias2) {
-#pragma unroll
-                                for (int q = 0; q < 32; q += 4) {
-                                    const float4 tb = __ldg((const float4*)(a.bias2 + co + q));
-                                    v[q] += tb.x; v[q + 1] += tb.y; v[q + 2] += tb.z; v[q + 3] += tb.w;
-                                }
-                            }
-                            if (OUT_MODE == 0) {
-#pragma unroll
-                                for (int c = 0; c < 8; ++c)
-                                    *(float4*)(orow + ((c ^ (m & 7)) << 4)) = make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 4; ++c)
-                                    *(uint4*)(orow + (((h * 4 + c) ^ (m & 7)) << 4)) =
-                                        make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
-                                                   pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
+                            for (int c = 0; c < 4; ++c) {
+                                const float4 t0 = bp[2 * c], t1 = bp[2 * c + 1];
+                                *(uint4*)(orow + (((h * 4 + c) ^ (lane & 7)) << 4)) =
+                                    make_uint4(pack_bf16(__uint_as_float(rc[8 * c]) + t0.x, __uint_as_float(rc[8 * c + 1]) + t0.y),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 2]) + t0.z, __uint_as_float(rc[8 * c + 3]) + t0.w),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 4]) + t1.x, __uint_as_float(rc[8 * c + 5]) + t1.y),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 6]) + t1.z, __uint_as_float(rc[8 * c + 7]) + t1.w));
                             }
                         }
-                        tr.mark(14);
-                        fence_proxy_async_smem();
-                        ok = __all_sync(0xffffffffu, epi_rendezvous());
-                        if (!ok) break;
-                        tr.mark(15);
-                        if (leader) {
-                            if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sidx * CS, tl.tx0, tl.ty0, tl.b);
-                            else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sidx * CS, tl.tx0, tl.ty0, tl.b);
-                            bulk_commit_group();
+                        if (p + 1 < NP) {
+                            tmem_ld_wait();
+                        } else if (last_tile) {                          // accumulators fully read: hand them back
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                        }
+                        if (h == PPS - 1) {
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                constexpr int CS = 32 * PPS;
+                                if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
+                                else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
+                                bulk_commit_group();
+                            }
                         }
                     }
+                    n_slice += NP / PPS;
                 }
+                t += cnt;
             }
-            t += cnt;
+            if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
         }
-        if (leader) bulk_wait_group<0>();                    // all stores have landed before the CTA retires
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
         if (lane == 0) {
@@ -442,9 +453,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         // one tile row (PW pixels) apart.  The tensor core applies the 128-byte swizzle to the
                         // absolute shared-memory address, so any 128-byte-aligned start works (base_offset 0).
                         const bool centre = second || a.ksize == 1;
-                        const int ky = centre ? 1 : tap / 3, kx = centre ? 1 : tap - 3 * (tap / 3);
+                        const int tap_pix = centre ? PW + 1 : tap + (PW - 3) * ((tap * 11) >> 5);   // ky * PW + kx
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
-                        uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (uint32_t)(ky * PW + kx) * 8;
+                        uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (uint32_t)tap_pix * 8;
                         const uint32_t acc = (kc | tap) != 0;
                         uint32_t td = tmem_d;
                         for (int slot = 0; slot < cnt; ++slot) {
@@ -593,23 +604,15 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     } else {
         memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
     }
-    if (bn >= 128) {      // half-height boxes for the two-CTA kernel
-        if (!encode_weights((CUtensorMap*)plan->tmap_half, a.w, a.Cin, taps * padded_cout(a.Cout), bn / 2)) return cudaErrorInvalidValue;
-        if (a.x2) {
-            if (!encode_weights((CUtensorMap*)plan->tmap2_half, a.w2, a.Cin2, a.Cout, bn / 2)) return cudaErrorInvalidValue;
-        } else {
-            memcpy(plan->tmap2_half, plan->tmap_half, sizeof(plan->tmap_half));
-        }
-    }
     if (!a.out_nchw) {
-        // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one 128-byte-wide slice of a tile
+        // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one epilogue warp's quarter (4 rows) of a 128-byte-wide slice of a tile
         EncodeTiledFn enc = get_encode_fn();
         if (!enc) return cudaErrorNotSupported;
         const bool ob = a.out_dtype == VD_BF16;
         const cuuint64_t es = ob ? 2 : 4;
         const cuuint64_t dims[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)std::max(a.B, 1)};
         const cuuint64_t strides[3] = {(cuuint64_t)a.Cout * es, (cuuint64_t)a.W * a.Cout * es, (cuuint64_t)a.H * a.W * a.Cout * es};
-        const cuuint32_t box[4] = {ob ? 64u : 32u, (cuuint32_t)TILE_W, (cuuint32_t)TILE_H, 1};
+        const cuuint32_t box[4] = {ob ? 64u : 32u, (cuuint32_t)TILE_W, 4, 1};      // one epilogue warp's rows
         const cuuint32_t estr[4] = {1, 1, 1, 1};
         if (enc((CUtensorMap*)plan->tmap_y, ob ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.y, dims,
                 strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -633,12 +636,6 @@ cudaError_t launch_conv_tc(const ConvArgs& a_in, const ConvTcPlan& plan, unsigne
     a.trace = g_conv_trace;
     if (!a.out_nchw && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
-    static const bool one_cta = getenv("VD_CONV_ONE_CTA") != nullptr;                        // timing studies
-    if (!one_cta && plan.bn >= 128 && conv_tc2_supported(a)) {
-        const cudaError_t e = launch_conv_tc2(a, plan, status, s);
-        if (e != cudaErrorNotSupported) return e;
-        (void)cudaGetLastError();
-    }
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2>(a, plan, status, s) : launch_one<16, false, 2>(a, plan, status, s);

@@ -55,10 +55,12 @@ __device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[
 
 struct Tile { int tx0, ty0, n0, b; };
 
-// Debug timeline: role r of this CTA appends (code << 48 | clock) records when a trace buffer is given.
+// Debug timeline (builds with -DVD_CONV_TRACE only): role r of this CTA appends (code << 48 | clock)
+// records when a trace buffer is given.
 struct Tracer {
     unsigned long long* p;
     int n;
+#ifdef VD_CONV_TRACE
     __device__ __forceinline__ void init(unsigned long long* base, int role) {
         p = base ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
         n = 0;
@@ -66,6 +68,10 @@ struct Tracer {
     __device__ __forceinline__ void mark(unsigned code) {
         if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFull);
     }
+#else   // production builds carry no tracing code at all (the MMA-issuing thread is latency critical)
+    __device__ __forceinline__ void init(unsigned long long*, int) {}
+    __device__ __forceinline__ void mark(unsigned) {}
+#endif
 };
 
 }  // namespace convtile

@@ -88,8 +88,6 @@ struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
     unsigned char tmap2[128];   // weights of the fused shortcut (copy of tmap when unused)
     unsigned char tmap_y[128];  // output tensor (NHWC outputs leave through bulk tensor stores)
-    unsigned char tmap_half[128];   // weights with half-height boxes (two-CTA kernel: each CTA stages BN/2 rows)
-    unsigned char tmap2_half[128];
     void* y;                    // the output address tmap_y was built for
     int batch;                  // frames covered by tmap_y
     int bn;
@@ -97,9 +95,6 @@ struct alignas(64) ConvTcPlan {
 };
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
-// two-CTA (cta_group::2) variant, conv_tc2.cu; launch_conv_tc routes to it where it applies
-bool conv_tc2_supported(const ConvArgs& a);
-cudaError_t launch_conv_tc2(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
 bool attn_tc_supported(const AttnArgs& a);
 size_t attn_tc_scratch_bytes(int B, int T, int C);
 cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
