@@ -143,11 +143,12 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
-    if (warp < NUM_PRODUCER_WARPS) {
+    if (warp < EPI_WARP0 && warp != MMA_WARP) {
         // ------------------------------------------------ operand prologue (producers)
         // The work is a flat sequence of units (item, chunk, tile slot); a unit's loads (three
         // 8-channel groups per thread, 480 threads) are all in flight before any is consumed.
-        const int j = tid & 7;                              // this thread's channel group within a chunk
+        const int ptid = (warp < MMA_WARP ? warp : warp - 1) * 32 + lane;   // 0..479 over the producer warps
+        const int j = ptid & 7;                             // this thread's channel group within a chunk
         const bool prologue = a.scale != nullptr;
         const bool silu = a.silu != 0;
         const int up = a.upsample ? 1 : 0;
@@ -163,7 +164,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             }
             if (p.t < sched.end) p.tile = sched.get(p.t + p.slot, BN);
         };
-        Tracer tr; tr.init(tid == 0 ? a.trace : nullptr, 0);
+        Tracer tr; tr.init(ptid == 0 ? a.trace : nullptr, 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         Pos cur;
@@ -179,7 +180,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             uint32_t vm = 0;
 #pragma unroll
             for (int u = 0; u < BATCH; ++u) {
-                const int pix = (u * NUM_PRODUCERS + tid) >> 3;
+                const int pix = (u * NUM_PRODUCERS + ptid) >> 3;
                 const int py = pix / PW, px = pix - py * PW;
                 const int oy = cur.tile.ty0 + py - 1, ox = cur.tile.tx0 + px - 1;
                 bool v = oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
@@ -226,7 +227,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
                 // row = halo pixel (128 B = 64 channels), 16-byte chunk c stored at c ^ (row & 7): the
                 // 128-byte swizzle of the K-major operand layout (tile bases are 1024-byte aligned)
-                const int pix = (u * NUM_PRODUCERS + tid) >> 3;
+                const int pix = (u * NUM_PRODUCERS + ptid) >> 3;
                 uint8_t* prow = dst_tile + pix * 128;
                 if (in_bf16) {
                     *(uint4*)(prow + ((j ^ (pix & 7)) << 4)) = make_uint4(o0, o1, o2, o3);
@@ -435,28 +436,29 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 tc_fence_after();
                 tr.mark(21);
                 const uint32_t tmem_d = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
+                uint32_t acc = 0;                             // the first MMA of an item overwrites the accumulator
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
-                    const bool second = kc >= kchunks;
-                    const int ntap = second ? 1 : taps;
+                    const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
+                    const int ntap = centre ? 1 : 9;
                     tr.mark(22);
                     ok = mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     tr.mark(23);
+                    // tap view: rows start (ky*PW + kx) pixels into the halo tile; eight-row groups are
+                    // one tile row (PW pixels) apart.  The tensor core applies the 128-byte swizzle to the
+                    // absolute shared-memory address, so any 128-byte-aligned start works (base_offset 0).
+                    const uint32_t a_chunk = a_lo0 + as * (A_STAGE_BYTES >> 4);
+                    uint32_t tap_off = centre ? (PW + 1) * 8 : 0;              // (ky*PW + kx) * 128 B >> 4
+                    int kx = 0;
                     for (int tap = 0; tap < ntap; ++tap) {
                         tr.mark(25);
                         ok = mbar_wait(smem_u32(&bars->b_full[bs]), bph, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         tr.mark(24);
-                        // tap view: rows start (ky*PW + kx) pixels into the halo tile; eight-row groups are
-                        // one tile row (PW pixels) apart.  The tensor core applies the 128-byte swizzle to the
-                        // absolute shared-memory address, so any 128-byte-aligned start works (base_offset 0).
-                        const bool centre = second || a.ksize == 1;
-                        const int tap_pix = centre ? PW + 1 : tap + (PW - 3) * ((tap * 11) >> 5);   // ky * PW + kx
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
-                        uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (uint32_t)tap_pix * 8;
-                        const uint32_t acc = (kc | tap) != 0;
+                        uint32_t a_lo = a_chunk + tap_off;
                         uint32_t td = tmem_d;
                         for (int slot = 0; slot < cnt; ++slot) {
                             umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
@@ -466,10 +468,12 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             a_lo += A_TILE_BYTES >> 4;
                             td += Cfg::ACC_COLS;
                         }
+                        acc = 1u;
                         // tcgen05.commit is served at a limited rate (about one per 700 cycles), so weight
                         // stages are handed back B_GROUP at a time
                         if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
                         if (++bs == Cfg::B_STAGES) { bs = 0; bph ^= 1; }
+                        if (++kx == 3) { kx = 0; tap_off += (PW - 2) * 8; } else tap_off += 8;
                     }
                     umma_commit(smem_u32(&bars->a_empty[as]));
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }

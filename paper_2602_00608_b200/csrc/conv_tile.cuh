@@ -18,9 +18,12 @@ constexpr int NUM_PRODUCER_WARPS = 15;
 constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // 480 = ITEMS / 3: three pairs per thread
 constexpr int BATCH = ITEMS / NUM_PRODUCERS;                         // 3
 static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the halo chunk exactly");
-constexpr int TMA_WARP = 15;
+// Warps map to the four SM sub-partitions by (warp % 4).  The MMA-issuing warp is latency critical
+// (the tensor pipe accepts little work ahead), so it shares its sub-partition with one producer
+// warp fewer than the others: producers are warps 0-11 and 13-15, warp 12 issues the MMAs.
+constexpr int MMA_WARP = 12;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
-constexpr int MMA_WARP = 20;
+constexpr int TMA_WARP = 20;
 constexpr int NUM_THREADS = 21 * 32;
 constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixels x 128 B: one output slice in smem
 
