@@ -84,6 +84,8 @@ attn_tc_kernel(const AttnTcParams a, const __grid_constant__ CUtensorMap tm_q, c
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
     const uint32_t tmem_o = tmem + 256;
+    griddep_launch();            // the next kernel may set itself up from here on
+    if (warp != 6) griddep_wait();   // every role but the MMA issue loop touches activations of earlier kernels
 
     if (warp < 4) {
         // ------------------------------------------------------------ softmax warps
@@ -297,6 +299,8 @@ attn_tc_kernel(const AttnTcParams a, const __grid_constant__ CUtensorMap tm_q, c
 // v [B][T][ld] -> vt [B][C][Tp] (tokens contiguous, zero beyond T)
 __global__ void transpose_v_kernel(const __nv_bfloat16* v, __nv_bfloat16* vt, int T, int Tp, int C, int ld) {
     __shared__ __nv_bfloat16 tile[32][33];
+    griddep_launch();
+    griddep_wait();
     const int b = blockIdx.z;
     const int t0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
     for (int i = threadIdx.y; i < 32; i += blockDim.y) {
@@ -353,8 +357,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status, cudaStream_t
     const int Tp = padded_tokens(a.T);
     {
         dim3 grid(Tp / 32, a.C / 32, a.B), block(32, 8);
-        transpose_v_kernel<<<grid, block, 0, s>>>((const __nv_bfloat16*)a.v, (__nv_bfloat16*)a.vt, a.T, Tp, a.C, a.ld_qkv);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_pdl(transpose_v_kernel, grid, block, 0, s, (const __nv_bfloat16*)a.v, (__nv_bfloat16*)a.vt, a.T, Tp, a.C, a.ld_qkv);
         if (e != cudaSuccess) return e;
     }
     CUtensorMap tq, tk, tv;
@@ -370,8 +373,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status, cudaStream_t
     }
     AttnTcParams p{a.o, a.B, a.T, a.C, a.ld_o, a.scale * 1.4426950408889634f};
     dim3 grid((a.T + BQ - 1) / BQ, a.C / DV, a.B);
-    attn_tc_kernel<<<grid, NUM_THREADS, SMEM_TOTAL, s>>>(p, tq, tk, tv, status);
-    return cudaGetLastError();
+    return launch_pdl(attn_tc_kernel, grid, dim3(NUM_THREADS), SMEM_TOTAL, s, p, tq, tk, tv, status);
 }
 
 }  // namespace vd

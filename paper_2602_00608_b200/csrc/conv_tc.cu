@@ -114,6 +114,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     Bars* bars = (Bars*)(smem_bias + Cfg::SMEM_BIAS);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
+    const long long t_entry = Tracer::now();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int taps = a.ksize * a.ksize;
     const int kchunks = a.Cin >> 6;
@@ -142,12 +143,17 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
+    // The kernel after this one may set itself up from here on.  Of this kernel, only the roles
+    // that touch activations wait for the kernel before it; weights (TMA warp) and the MMA issue
+    // loop (fed by the other roles) need no wait.
+    griddep_launch();
 
-    if (warp < EPI_WARP0 && warp != MMA_WARP) {
+    if (is_producer_warp(warp)) {
+        griddep_wait();
         // ------------------------------------------------ operand prologue (producers)
         // The work is a flat sequence of units (item, chunk, tile slot); a unit's loads (three
         // 8-channel groups per thread, 480 threads) are all in flight before any is consumed.
-        const int ptid = (warp < MMA_WARP ? warp : warp - 1) * 32 + lane;   // 0..479 over the producer warps
+        const int ptid = producer_index(warp) * 32 + lane;  // 0..479 over the producer warps
         const int j = ptid & 7;                             // this thread's channel group within a chunk
         const bool prologue = a.scale != nullptr;
         const bool silu = a.silu != 0;
@@ -251,6 +257,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         // Each warp owns a quarter of the accumulator rows (32 pixels = four rows of the 16x8 tile)
         // and works on its own: no synchronisation between the four warps.  TMEM reads are issued
         // one column block ahead of the one being processed.
+        griddep_wait();
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
         const bool reduce_add = a.residual != nullptr;       // y is the residual stream: the tile is added into it
         Tracer tr; tr.init(tid == EPI_WARP0 * 32 ? a.trace : nullptr, 2);
@@ -377,6 +384,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 t += cnt;
             }
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
+            tr.mark(12);
         }
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
@@ -424,6 +432,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
             const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)), b_lo0 = desc_lo(smem_u32(smem_b));
             Tracer tr; tr.init(a.trace, 1);
+            tr.mark_at(40, t_entry);
+            tr.mark(41);
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
             bool ok = true;
             int n_item = 0;
@@ -452,11 +462,11 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     uint32_t tap_off = centre ? (PW + 1) * 8 : 0;              // (ky*PW + kx) * 128 B >> 4
                     int kx = 0;
                     for (int tap = 0; tap < ntap; ++tap) {
-                        tr.mark(25);
+                        tr.mark_fine(25);
                         ok = mbar_wait(smem_u32(&bars->b_full[bs]), bph, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        tr.mark(24);
+                        tr.mark_fine(24);
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
                         uint32_t a_lo = a_chunk + tap_off;
                         uint32_t td = tmem_d;
@@ -564,9 +574,8 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
     int grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
     if (getenv("VD_CONV_GRID")) grid = std::min(grid, atoi(getenv("VD_CONV_GRID")));   // timing studies
-    kern<<<grid, NUM_THREADS, TileCfg<BN>::SMEM_TOTAL, s>>>(a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
-                                                            *(const CUtensorMap*)plan.tmap_y, status);
-    return cudaGetLastError();
+    return launch_pdl(kern, dim3(grid), dim3(NUM_THREADS), TileCfg<BN>::SMEM_TOTAL, s, a, *(const CUtensorMap*)plan.tmap,
+                      *(const CUtensorMap*)plan.tmap2, *(const CUtensorMap*)plan.tmap_y, status);
 }
 
 }  // namespace

@@ -18,13 +18,19 @@ constexpr int NUM_PRODUCER_WARPS = 15;
 constexpr int NUM_PRODUCERS = NUM_PRODUCER_WARPS * 32;               // 480 = ITEMS / 3: three pairs per thread
 constexpr int BATCH = ITEMS / NUM_PRODUCERS;                         // 3
 static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the halo chunk exactly");
-// Warps map to the four SM sub-partitions by (warp % 4).  The MMA-issuing warp is latency critical
-// (the tensor pipe accepts little work ahead), so it shares its sub-partition with one producer
-// warp fewer than the others: producers are warps 0-11 and 13-15, warp 12 issues the MMAs.
-constexpr int MMA_WARP = 12;
+// Warps map to the four SM sub-partitions by (warp % 4), and a sub-partition's scheduler gives the
+// MMA-issuing thread no priority: measured, fifteen warps of dense arithmetic stretch its
+// wait / 4 x MMA / commit sequence from 513 to about 1800 cycles, while the same warps kept off its
+// sub-partition cost nothing.  So sub-partition 0 carries only the MMA warp, the TMA warp and one
+// epilogue warp (warps 8, 12 and 20 idle until the end), and the fifteen producer warps are the
+// warps with warp % 4 != 0 outside the epilogue: five per remaining sub-partition.
+constexpr int MMA_WARP = 0;
+constexpr int TMA_WARP = 4;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
-constexpr int TMA_WARP = 20;
-constexpr int NUM_THREADS = 21 * 32;
+constexpr int NUM_THREADS = 24 * 32;
+__device__ __forceinline__ bool is_producer_warp(int warp) { return (warp & 3) != 0 && (warp < EPI_WARP0 || warp >= EPI_WARP0 + 4); }
+// 0..14 over the producer warps
+__device__ __forceinline__ int producer_index(int warp) { return (warp < EPI_WARP0 ? (warp >> 2) : 4) * 3 + (warp & 3) - 1; }
 constexpr int OUT_SLICE_BYTES = 128 * 128;                           // 128 pixels x 128 B: one output slice in smem
 
 struct Raw8 { uint4 lo, hi; };   // eight channels of one pixel: bf16 -> lo only; fp32 -> lo + hi
@@ -64,16 +70,28 @@ struct Tracer {
     unsigned long long* p;
     int n;
 #ifdef VD_CONV_TRACE
+    // VD_CONV_TRACE is a mask of the roles that record (bit = role number), so that one role can
+    // be observed while the others run the production code
     __device__ __forceinline__ void init(unsigned long long* base, int role) {
-        p = base ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
+        p = (base && ((VD_CONV_TRACE >> role) & 1)) ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
         n = 0;
     }
     __device__ __forceinline__ void mark(unsigned code) {
         if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFull);
     }
+    __device__ __forceinline__ void mark_fine(unsigned code) {       // per-tap marks of the MMA thread: bit 4 of the mask
+        if ((VD_CONV_TRACE >> 4) & 1) mark(code);
+    }
+    __device__ __forceinline__ void mark_at(unsigned code, long long clk) {
+        if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clk & 0xFFFFFFFFFFFFull);
+    }
+    static __device__ __forceinline__ long long now() { return clock64(); }
 #else   // production builds carry no tracing code at all (the MMA-issuing thread is latency critical)
     __device__ __forceinline__ void init(unsigned long long*, int) {}
     __device__ __forceinline__ void mark(unsigned) {}
+    __device__ __forceinline__ void mark_fine(unsigned) {}
+    __device__ __forceinline__ void mark_at(unsigned, long long) {}
+    static __device__ __forceinline__ long long now() { return 0; }
 #endif
 };
 

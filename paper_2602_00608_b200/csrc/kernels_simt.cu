@@ -30,6 +30,8 @@ __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + expf(-v));
 // hit branch) and writes z and the new motion vector back in the latents' own layout/dtype.
 template <typename T>
 __global__ void ingest_kernel(IngestArgs a) {
+    griddep_launch();
+    griddep_wait();
     const int64_t total = (int64_t)a.B * a.C * a.h * a.w;
     const T* z = (const T*)a.z;
     const T* vp = (const T*)a.v_prev;
@@ -54,24 +56,14 @@ __global__ void ingest_kernel(IngestArgs a) {
 }
 
 // ------------------------------------------------------------------------------ GroupNorm stats
-// Pass A: every block reduces a run of pixels of one sample to per-group (count, mean, M2).
-// A thread owns one 4-channel slot (inside one group, since C/G is a multiple of 4) and walks
-// down the pixels; sums are taken about the first value seen, so a large common offset does
-// not cancel; partial results are merged with the parallel-variance (Chan) update.
-struct Moments { float n, mean, m2; };
-__device__ __forceinline__ Moments merge(Moments a, Moments b) {
-    if (b.n == 0.f) return a;
-    if (a.n == 0.f) return b;
-    const float n = a.n + b.n;
-    const float d = b.mean - a.mean;
-    const float f = b.n / n;
-    Moments r;
-    r.n = n;
-    r.mean = fmaf(d, f, a.mean);
-    r.m2 = a.m2 + b.m2 + d * d * a.n * f;
-    return r;
-}
-
+// One launch.  Every block reduces a run of pixels of one sample to per-group sums of (x - K) and
+// (x - K)^2, where K is a reference value per (sample, group) that every block reads from the same
+// place (the mean of the group's first four channels at the sample's centre pixel), so the sums
+// of different blocks add without correction terms and a large common offset does not cancel.
+// A thread owns one 4-channel slot (inside one group, since C/G is a multiple of 4) and walks down
+// the pixels.  The block that arrives last for its sample adds the records of all blocks in a
+// fixed order and writes scale and shift; the order of every sum is fixed by the sizes alone, so
+// the result is bitwise reproducible and independent of the batch a sample is decoded in.
 template <typename T> __device__ __forceinline__ void load4(const T* p, float v[4]);
 template <> __device__ __forceinline__ void load4<float>(const float* p, float v[4]) {
     const float4 t = __ldg((const float4*)p);
@@ -83,125 +75,127 @@ template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bflo
     v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
 }
 
-constexpr int kGnThreads = 256;
+constexpr int kGnThreads = 512;
+constexpr int kGnFinalLoads = (kGnMaxChunks + 15) / 16;   // records per lane when 16 lanes share a group
 
-template <typename T>
-__global__ void __launch_bounds__(kGnThreads) gn_partial_kernel(GnArgs a, int chunks, int pix_per_chunk) {
-    __shared__ Moments sm[kGnThreads];
+template <typename T, int U>
+__global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int chunks, int pix_per_chunk) {
+    __shared__ float2 sm[kGnThreads];
+    __shared__ int s_last;
+    griddep_launch();
+    griddep_wait();
     const int n = blockIdx.y;
     const int chunk = blockIdx.x;
-    const int slots = a.C / 4;                       // 4-channel slots per pixel (<= 128... or more: loop)
+    const int slots = a.C / 4;                       // 4-channel slots per pixel (<= kGnThreads)
     const int p0 = chunk * pix_per_chunk;
     const int p1 = min(a.P, p0 + pix_per_chunk);
     const T* x = (const T*)a.x + (size_t)n * a.P * a.C;
     const int cpg = a.C / a.G;
+    const int rows = kGnThreads / slots;             // pixels handled side by side
+    const int slot = threadIdx.x % slots;
+    const int row = threadIdx.x / slots;
 
-    // slot loop: when C/4 > blockDim (not the case for C <= 1024) a thread would own several slots
-    for (int slot0 = 0; slot0 < slots; slot0 += kGnThreads) {
-        const int lanes = min(slots - slot0, kGnThreads);       // threads across the channel axis
-        const int rows = kGnThreads / lanes;                    // pixels handled side by side
-        const int slot = slot0 + (threadIdx.x % lanes);
-        const int row = threadIdx.x / lanes;
-        Moments m = {0.f, 0.f, 0.f};
-        if (row < rows && p0 + row < p1) {
-            float v[4];
-            load4<T>(x + (size_t)(p0 + row) * a.C + slot * 4, v);
-            const float k = v[0];
-            float s = 0.f, ss = 0.f, cnt = 0.f;
-            int p = p0 + row;
-            for (; p + 3 * rows < p1; p += 4 * rows) {
-                float u[4][4];
+    float s = 0.f, ss = 0.f;
+    if (row < rows && p0 + row < p1) {
+        float kv[4];
+        load4<T>(x + (size_t)(a.P / 2) * a.C + (slot * 4 / cpg) * cpg, kv);
+        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
+        int p = p0 + row;
+        for (; p + (U - 1) * rows < p1; p += U * rows) {        // U independent loads in flight
+            float u[U][4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) load4<T>(x + (size_t)(p + j * rows) * a.C + slot * 4, u[j]);
+            for (int j = 0; j < U; ++j) load4<T>(x + (size_t)(p + j * rows) * a.C + slot * 4, u[j]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float d = u[j][e] - k;
-                        s += d;
-                        ss = fmaf(d, d, ss);
-                    }
-                cnt += 16.f;
-            }
-            for (; p < p1; p += rows) {
-                load4<T>(x + (size_t)p * a.C + slot * 4, v);
+            for (int j = 0; j < U; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float d = v[e] - k;
+                    const float d = u[j][e] - k;
                     s += d;
                     ss = fmaf(d, d, ss);
                 }
-                cnt += 4.f;
-            }
-            const float md = s / cnt;
-            m.n = cnt;
-            m.mean = k + md;
-            m.m2 = fmaxf(ss - s * md, 0.f);
         }
-        sm[threadIdx.x] = m;
-        __syncthreads();
-        // one thread per group present in this slot window gathers its members
-        const int g_lo = (slot0 * 4) / cpg;
-        const int g_hi = ((slot0 + lanes) * 4 - 1) / cpg;
-        const int g = g_lo + threadIdx.x;
-        if (g <= g_hi) {
-            const int s_lo = max(g * cpg / 4 - slot0, 0);
-            const int s_hi = min((g + 1) * cpg / 4 - slot0, lanes);
-            Moments acc = {0.f, 0.f, 0.f};
-            for (int r = 0; r < rows; ++r)
-                for (int sl = s_lo; sl < s_hi; ++sl) acc = merge(acc, sm[r * lanes + sl]);
-            float* out = a.partial + (((size_t)n * kGnMaxChunks + chunk) * a.G + g) * 4;
-            if (slot0 > 0 && (slot0 * 4) % cpg != 0 && g == g_lo) {
-                // group straddles two slot windows: fold into what the previous window wrote
-                Moments prev = {out[0], out[1], out[2]};
-                acc = merge(prev, acc);
+        for (; p < p1; p += rows) {
+            float v[4];
+            load4<T>(x + (size_t)p * a.C + slot * 4, v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float d = v[e] - k;
+                s += d;
+                ss = fmaf(d, d, ss);
             }
-            out[0] = acc.n; out[1] = acc.mean; out[2] = acc.m2;
         }
-        __syncthreads();
     }
-}
-
-// Pass B: one block per (group, sample) merges that group's chunk partials (independent loads
-// first, then a fixed-order tree), and folds the statistics with the affine parameters into
-// per-(sample, channel) scale and shift.
-constexpr int kGnFinalThreads = 128;
-__global__ void __launch_bounds__(kGnFinalThreads) gn_finalize_kernel(GnArgs a, int chunks) {
-    __shared__ Moments sm[kGnFinalThreads / 32];
-    const int g = blockIdx.x, n = blockIdx.y;
-    const int cpg = a.C / a.G;
-    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    constexpr int PER = kGnMaxChunks / kGnFinalThreads;          // 8 partials per thread at most
-    float4 p[PER];
-#pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        const int k = threadIdx.x + i * kGnFinalThreads;
-        p[i] = (k < chunks) ? *(const float4*)(a.partial + (((size_t)n * kGnMaxChunks + k) * a.G + g) * 4)
-                            : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    Moments m = {0.f, 0.f, 0.f};
-#pragma unroll
-    for (int i = 0; i < PER; ++i) m = merge(m, Moments{p[i].x, p[i].y, p[i].z});
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        Moments o;
-        o.n = __shfl_down_sync(0xffffffffu, m.n, d);
-        o.mean = __shfl_down_sync(0xffffffffu, m.mean, d);
-        o.m2 = __shfl_down_sync(0xffffffffu, m.m2, d);
-        m = merge(m, o);
-    }
-    if (lane == 0) sm[warp] = m;
+    sm[threadIdx.x] = make_float2(s, ss);
     __syncthreads();
-    Moments t = sm[0];
-#pragma unroll
-    for (int w = 1; w < kGnFinalThreads / 32; ++w) t = merge(t, sm[w]);
-    const float rstd = (float)(1.0 / sqrt((double)t.m2 / (double)t.n + (double)a.eps));
-    for (int cc = threadIdx.x; cc < cpg; cc += kGnFinalThreads) {
-        const int c = g * cpg + cc;
-        const float sc = a.gamma[c] * rstd;
-        a.scale[(size_t)n * a.C + c] = sc;
-        a.shift[(size_t)n * a.C + c] = a.beta[c] - t.mean * sc;
+    // one thread per group adds its members: rows x (slots of the group), in a fixed order
+    if (threadIdx.x < a.G) {
+        const int g = threadIdx.x;
+        const int spg = cpg / 4;
+        float2 acc = make_float2(0.f, 0.f);
+        for (int r = 0; r < rows; ++r)
+            for (int sl = g * spg; sl < (g + 1) * spg; ++sl) {
+                const float2 v = sm[r * slots + sl];
+                acc.x += v.x;
+                acc.y += v.y;
+            }
+        ((float2*)a.partial)[((size_t)n * kGnMaxChunks + chunk) * a.G + g] = acc;
     }
+    __syncthreads();
+
+    // The block of this sample that finishes last folds the records into scale and shift.
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(a.counters + n, 1u);
+        s_last = (prev == (unsigned int)chunks - 1u) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    int tpg = 16;                                    // lanes cooperating on one group (a power of two)
+    while (tpg * a.G > kGnThreads && tpg > 1) tpg >>= 1;
+    const int sub = threadIdx.x % tpg;
+    const float inv_n = 1.f / ((float)a.P * (float)cpg);
+    for (int g0 = 0; g0 < a.G; g0 += kGnThreads / tpg) {        // uniform trip count: every lane reaches the shuffles
+        const bool valid = g0 + threadIdx.x / tpg < a.G;
+        const int g = valid ? g0 + threadIdx.x / tpg : a.G - 1;
+        const int nrec = valid ? chunks : 0;
+        const float2* rec = (const float2*)a.partial + (size_t)n * kGnMaxChunks * a.G + g;
+        // loads that do not depend on the records go first, so one memory round trip covers them all
+        float kv[4];
+        load4<T>(x + (size_t)(a.P / 2) * a.C + g * cpg, kv);
+        const int c0 = g * cpg + min(sub, cpg - 1);
+        const float gamma0 = __ldg(a.gamma + c0), beta0 = __ldg(a.beta + c0);
+        float2 acc = make_float2(0.f, 0.f);
+        for (int k0 = sub; k0 < nrec; k0 += kGnFinalLoads * tpg) {
+            float2 r[kGnFinalLoads];
+#pragma unroll
+            for (int i = 0; i < kGnFinalLoads; ++i) {
+                const int k = k0 + i * tpg;
+                r[i] = (k < nrec) ? __ldcg(rec + (size_t)k * a.G) : make_float2(0.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < kGnFinalLoads; ++i) {
+                acc.x += r[i].x;
+                acc.y += r[i].y;
+            }
+        }
+        for (int d = tpg >> 1; d > 0; d >>= 1) {     // a + b == b + a: both lanes of a pair end with equal values
+            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, d);
+            acc.y += __shfl_xor_sync(0xffffffffu, acc.y, d);
+        }
+        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
+        const float md = acc.x * inv_n;
+        const float var = fmaxf(fmaf(-md, md, acc.y * inv_n), 0.f);
+        const float mean = k + md;
+        const float rstd = 1.f / sqrtf(var + a.eps);
+        for (int cc = sub; valid && cc < cpg; cc += tpg) {
+            const int c = g * cpg + cc;
+            const float sc = (cc == sub ? gamma0 : a.gamma[c]) * rstd;
+            a.scale[(size_t)n * a.C + c] = sc;
+            a.shift[(size_t)n * a.C + c] = (cc == sub ? beta0 : a.beta[c]) - mean * sc;
+        }
+    }
+    if (threadIdx.x == 0) a.counters[n] = 0u;        // ready for the next launch
 }
 
 // ------------------------------------------------------------------------------- direct conv
@@ -211,6 +205,8 @@ constexpr int KC = 8;
 
 template <typename TIn, typename TOut, int TH, int TW, int PPT, int CPT, int CGROUPS>
 __global__ void __launch_bounds__((TH * TW / PPT) * CGROUPS) conv_simt_kernel(ConvArgs a) {
+    griddep_launch();
+    griddep_wait();
     constexpr int NPG = TH * TW / PPT;
     constexpr int CT = CPT * CGROUPS;
     constexpr int NT = NPG * CGROUPS;
@@ -301,11 +297,11 @@ cudaError_t conv_simt_dispatch(const ConvArgs& a, cudaStream_t s) {
     if (a.Cout <= 8) {
         constexpr int TH = 16, TW = 16, CT = 4;
         dim3 grid(((a.W + TW - 1) / TW) * ((a.H + TH - 1) / TH), (a.Cout + CT - 1) / CT, a.B);
-        conv_simt_kernel<TIn, TOut, TH, TW, 1, 4, 1><<<grid, 256, 0, s>>>(a);
+        launch_pdl(conv_simt_kernel<TIn, TOut, TH, TW, 1, 4, 1>, grid, dim3(256), 0, s, a);
     } else {
         constexpr int TH = 8, TW = 8, CT = 64;
         dim3 grid(((a.W + TW - 1) / TW) * ((a.H + TH - 1) / TH), (a.Cout + CT - 1) / CT, a.B);
-        conv_simt_kernel<TIn, TOut, TH, TW, 4, 4, 16><<<grid, 256, 0, s>>>(a);
+        launch_pdl(conv_simt_kernel<TIn, TOut, TH, TW, 4, 4, 16>, grid, dim3(256), 0, s, a);
     }
     return cudaGetLastError();
 }
@@ -317,6 +313,8 @@ constexpr int kAttnQ = 8, kAttnKeys = 32;
 
 template <typename T>
 __global__ void __launch_bounds__(kAttnQ * 32) attn_simt_kernel(AttnArgs a) {
+    griddep_launch();
+    griddep_wait();
     extern __shared__ float smem[];
     const int C = a.C;
     float* s_q = smem;                               // [kAttnQ][C]
@@ -413,22 +411,20 @@ int grid_for(int64_t n, int threads) {
 
 cudaError_t launch_ingest(const IngestArgs& a, cudaStream_t s) {
     const int64_t n = (int64_t)a.B * a.C * a.h * a.w;
-    if (a.dtype == VD_BF16) ingest_kernel<__nv_bfloat16><<<grid_for(n, 256), 256, 0, s>>>(a);
-    else ingest_kernel<float><<<grid_for(n, 256), 256, 0, s>>>(a);
+    if (a.dtype == VD_BF16) launch_pdl(ingest_kernel<__nv_bfloat16>, dim3(grid_for(n, 256)), dim3(256), 0, s, a);
+    else launch_pdl(ingest_kernel<float>, dim3(grid_for(n, 256)), dim3(256), 0, s, a);
     return cudaGetLastError();
 }
 
 cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s) {
+    if (a.C % 4 != 0 || a.C / 4 > kGnThreads || a.G > kGnThreads || (a.C / a.G) % 4 != 0) return cudaErrorInvalidValue;
     // chunks per sample depend on the sample size only (so a frame's statistics, and with them
     // the frame, do not depend on the batch it is decoded in): at least 32 pixels per chunk
     int ppc = max(32, (a.P + kGnMaxChunks - 1) / kGnMaxChunks);
     int chunks = (a.P + ppc - 1) / ppc;
     dim3 grid(chunks, a.B);
-    if (a.dtype == VD_BF16) gn_partial_kernel<__nv_bfloat16><<<grid, kGnThreads, 0, s>>>(a, chunks, ppc);
-    else gn_partial_kernel<float><<<grid, kGnThreads, 0, s>>>(a, chunks, ppc);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    gn_finalize_kernel<<<dim3(a.G, a.B), kGnFinalThreads, 0, s>>>(a, chunks);
+    if (a.dtype == VD_BF16) launch_pdl(gn_stats_kernel<__nv_bfloat16, 16>, grid, dim3(kGnThreads), 0, s, a, chunks, ppc);
+    else launch_pdl(gn_stats_kernel<float, 8>, grid, dim3(kGnThreads), 0, s, a, chunks, ppc);
     return cudaGetLastError();
 }
 
@@ -448,11 +444,11 @@ cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s) {
     if (a.dtype == VD_BF16) {
         e = cudaFuncSetAttribute(attn_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attn_simt_kernel<__nv_bfloat16><<<grid, kAttnQ * 32, smem, s>>>(a);
+        launch_pdl(attn_simt_kernel<__nv_bfloat16>, grid, dim3(kAttnQ * 32), smem, s, a);
     } else {
         e = cudaFuncSetAttribute(attn_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        attn_simt_kernel<float><<<grid, kAttnQ * 32, smem, s>>>(a);
+        launch_pdl(attn_simt_kernel<float>, grid, dim3(kAttnQ * 32), smem, s, a);
     }
     return cudaGetLastError();
 }
@@ -482,14 +478,14 @@ cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cud
 // allocator is simply off limits (inside a host callback, after a memory budget was frozen).
 // For them the chunk partials of the reduction live in the fixed device array below instead of a
 // buffer passed in.  The price is a size limit and shared state: every GPU that loads this
-// library carries the array (1 MiB) until the process exits, and all calls on a device use the
+// library carries the array (148 KiB) until the process exits, and all calls on a device use the
 // same array, so two calls whose kernels can overlap on the GPU (different streams, no ordering
-// between them) race on it.  Nothing in the array has to start at zero: every slot the second
-// kernel reads was written by the first kernel of the same call, so stale contents of an earlier
-// call are never observed.
+// between them) race on it.  The chunk records need no clearing (every record read was written
+// by the same call); the arrival counters behind them must start at zero and are cleared by an
+// asynchronous memset at the start of every call.
 namespace {
 constexpr int kStaticGnMaxBatchTimesGroups = 64;     // e.g. 2 frames x 32 groups, or 8 x 8
-static __device__ __align__(256) float g_gn_static_partial[kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 4];   // 1 MiB
+static __device__ __align__(256) float g_gn_static_partial[kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2 + 64];   // 148 KiB of chunk records + 64 arrival counters
 
 std::mutex g_static_mu;
 constexpr int kMaxDevices = 64;
@@ -535,8 +531,11 @@ extern "C" VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, 
     float* partial = nullptr;
     cudaError_t e = static_scratch_of_current_device(&partial);
     if (e == cudaSuccess) {
-        GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial};
-        e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
+        // the arrival counters live behind the records; they must be zero when the kernel starts
+        unsigned int* counters = (unsigned int*)(partial + (size_t)kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2);
+        e = cudaMemsetAsync(counters, 0, 64 * sizeof(unsigned int), (cudaStream_t)cuda_stream);
+        GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial, counters};
+        if (e == cudaSuccess) e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
     }
     if (e != cudaSuccess) {
         set_last_error((std::string("vd_op_gn_stats_static: ") + cudaGetErrorString(e)).c_str());

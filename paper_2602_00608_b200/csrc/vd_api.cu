@@ -49,7 +49,7 @@ struct vd_handle_s {
     std::vector<WeightJob> jobs;
     std::string err;
     int stop_after = -1;
-    size_t status_off = 0, lat_stage_off = 0, frm_stage_off = 0;
+    size_t status_off = 0, lat_stage_off = 0, frm_stage_off = 0, gn_counter_off = 0;
     size_t total = 0;
 };
 
@@ -105,9 +105,10 @@ class Planner {
         Step s{};
         s.kind = VD_STEP_GN_STATS;
         s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
-                      ptr<float>(b_off), ptr<float>(scale_off_), ptr<float>(shift_off_), ptr<float>(partial_off_)};
+                      ptr<float>(b_off), ptr<float>(scale_off_), ptr<float>(shift_off_), ptr<float>(partial_off_),
+                      ptr<unsigned int>(partial_off_ + gn_partial_bytes(cfg_.max_batch, cfg_.norm_groups))};
         fill_info(s, name, 0, C, C, 0, 0, H, W, C, VD_F32, 0, -1);
-        s.info.launches = 2;
+        s.info.launches = 1;
         s.info.bytes_per_frame = (double)H * W * C * elt(dtype);
         h_->steps.push_back(s);
     }
@@ -264,6 +265,7 @@ class Planner {
         scale_off_ = scale_buf_[0];
         shift_off_ = shift_buf_[0];
         partial_off_ = alloc(vd_gn_scratch_bytes(B, cfg_.norm_groups));
+        h_->gn_counter_off = partial_off_ + gn_partial_bytes(B, cfg_.norm_groups);
         zbuf_ = alloc((size_t)B * P0 * lc * 4);
         xs_[0] = alloc((size_t)B * max_x * 4);
         xs_[1] = alloc((size_t)B * max_x * 4);
@@ -405,6 +407,20 @@ cudaError_t launch_step(const vd_handle_s* h, const Step& st, int B, const void*
     return cudaErrorInvalidValue;
 }
 
+}  // namespace
+
+namespace vd {
+static thread_local bool t_pdl_active = false;
+bool pdl_enabled() {
+    static const bool off = getenv("VD_NO_PDL") != nullptr;
+    return t_pdl_active && !off;
+}
+PdlScope::PdlScope(bool on) : prev(t_pdl_active) { t_pdl_active = on; }
+PdlScope::~PdlScope() { t_pdl_active = prev; }
+}  // namespace vd
+
+namespace {
+
 vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, float lambda, void* z_out, void* v_out,
                       void* frames, int32_t batch, void* stream, float* ms, int n_ms) {
     if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
@@ -424,6 +440,7 @@ vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, floa
         }
         cudaEventRecord(ev[0], s);
     }
+    PdlScope pdl(true);
     for (int i = 0; i < n; ++i) {
         cudaError_t e = launch_step(h, h->steps[i], batch, latents, v_prev, lambda, z_out, v_out, frames, s);
         if (e != cudaSuccess) {
@@ -495,6 +512,8 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
     }
     cudaStream_t s = (cudaStream_t)cuda_stream;
     e = cudaMemsetAsync(h->ws + h->status_off, 0, 256, s);
+    // arrival counters of the GroupNorm statistics kernel: zero once, every launch leaves them zero
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + h->gn_counter_off, 0, (size_t)cfg->max_batch * 4, s);
     if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "status memset"); }
     for (const WeightJob& j : h->jobs) {
         const vd_tensor* t = find_tensor(weights, n_weights, j.name);
@@ -706,7 +725,7 @@ vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* w_packe
 
 size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups) {
     if (batch < 1 || groups < 1) return 0;
-    return (size_t)batch * kGnMaxChunks * groups * 4 * sizeof(float);
+    return gn_scratch_bytes(batch, groups);
 }
 
 vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w, int32_t c, int32_t groups,
@@ -717,8 +736,10 @@ vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h,
     if (batch < 0 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups != 0 || (c / groups) % 4 != 0 || c > 1024)
         return fail(nullptr, VD_ERR_INVALID_ARG, "bad GroupNorm sizes (groups must hold a multiple of 4 channels)");
     if (batch == 0) return VD_OK;
-    GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch};
-    cudaError_t e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
+    unsigned int* counters = (unsigned int*)((char*)scratch + gn_partial_bytes(batch, groups));
+    GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch, counters};
+    cudaError_t e = cudaMemsetAsync(counters, 0, (size_t)batch * sizeof(unsigned int), (cudaStream_t)cuda_stream);
+    if (e == cudaSuccess) e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_gn_stats");
 }
 

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "vd.h"
 
 namespace vd {
@@ -40,9 +42,13 @@ struct GnArgs {
     const float* beta;      // [C]
     float* scale;           // [B,C]
     float* shift;           // [B,C]
-    float* partial;         // [B, kGnMaxChunks, G, 4] scratch
+    float* partial;         // [B, kGnMaxChunks, G, 2] scratch
+    unsigned int* counters; // [B] arrival counters, zero before the launch; the kernel leaves them zero
 };
-constexpr int kGnMaxChunks = 1024;
+constexpr int kGnMaxChunks = 296;      // two blocks per SM on a 148-SM device
+// bytes of the partial records / of the whole scratch (records, then the arrival counters)
+inline size_t gn_partial_bytes(int B, int G) { return (size_t)B * kGnMaxChunks * G * 2 * sizeof(float); }
+inline size_t gn_scratch_bytes(int B, int G) { return gn_partial_bytes(B, G) + (((size_t)B * 4 + 255) / 256) * 256; }
 
 struct AttnArgs {
     const void* q; const void* k; const void* v; void* o;
@@ -67,7 +73,7 @@ void set_last_error(const char* msg);
 
 // ---- FFMA kernels (kernels_simt.cu)
 cudaError_t launch_ingest(const IngestArgs& a, cudaStream_t s);
-cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s);          // two launches
+cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s);          // one launch (the last block per sample finalises)
 cudaError_t launch_conv_simt(const ConvArgs& a, cudaStream_t s);
 cudaError_t launch_attn_simt(const AttnArgs& a, cudaStream_t s);
 // OIHW (or [out,in]) weight of dtype `w_dtype` -> fp32 [tap][Cin][Cout]
@@ -98,5 +104,43 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
 bool attn_tc_supported(const AttnArgs& a);
 size_t attn_tc_scratch_bytes(int B, int T, int C);
 cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
+
+
+// ---- programmatic dependent launch
+// Every kernel of the decode path is launched so that its blocks may become resident while the
+// kernel before it in the stream is still draining: they set themselves up (barriers, tensor
+// memory, weight prefetch), then griddep_wait() returns once the preceding kernel has completed
+// and its writes are visible.  Rules that make the chain safe: (1) every such kernel executes
+// griddep_wait() in at least one thread before it exits, so "kernel N completed" implies "all
+// kernels before N completed"; (2) nothing a predecessor writes is read, and nothing it reads is
+// written, before the wait.
+// Dependent launches are used only inside a PdlScope (the decode loop): the single-operator entry
+// points launch plainly, since their inputs may come from work this library knows nothing about.
+bool pdl_enabled();     // inside a PdlScope, and the environment variable VD_NO_PDL is not set
+struct PdlScope {
+    explicit PdlScope(bool on);
+    ~PdlScope();
+    bool prev;
+};
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
 
 }  // namespace vd
