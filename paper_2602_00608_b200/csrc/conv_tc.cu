@@ -131,9 +131,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     sched.pair = PAIR;
 
     if (tid == 0) {
-        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), 1); }
-        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
+        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), PAIR); }
+        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), PAIR); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), PAIR); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -151,106 +151,142 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     if (is_producer_warp(warp)) {
         griddep_wait();
         // ------------------------------------------------ operand prologue (producers)
-        // The work is a flat sequence of units (item, chunk, tile slot); a unit's loads (three
-        // 8-channel groups per thread, 480 threads) are all in flight before any is consumed.
+        // The work is a sequence of units (item, chunk, tile slot); a thread owns three (pixel,
+        // 8-channel group) entries of every unit, all loaded before any is consumed.  The role is
+        // bound by instruction issue, so whatever depends only on the thread (where an entry sits
+        // in the halo tile, in shared memory and relative to the tile's first source pixel) is
+        // computed once, and tiles whose halo lies inside the image skip the bounds checks.
         const int ptid = producer_index(warp) * 32 + lane;  // 0..479 over the producer warps
         const int j = ptid & 7;                             // this thread's channel group within a chunk
         const bool prologue = a.scale != nullptr;
         const bool silu = a.silu != 0;
         const int up = a.upsample ? 1 : 0;
-        struct Pos { int t, cnt, kc, slot; Tile tile; };
-        auto advance = [&](Pos& p) {
-            if (++p.slot == p.cnt) {
-                p.slot = 0;
-                if (++p.kc == ktotal) {
-                    p.kc = 0;
-                    p.t += p.cnt;
-                    if (p.t < sched.end) p.cnt = sched.count(p.t);
-                }
-            }
-            if (p.t < sched.end) p.tile = sched.get(p.t + p.slot, BN);
-        };
+        constexpr int ESZ = IN_BF16 ? 2 : 4;
+        uint32_t soff[BATCH];        // byte offset of the entry's (first) 8/16-byte store within a tile chunk
+        int goff[BATCH];             // byte offset of the entry's source pixel from the tile's first source pixel
+        uint32_t pyx[BATCH];         // py | px << 8 | (entry lies in the tile proper, not the halo) << 16
+#pragma unroll
+        for (int u = 0; u < BATCH; ++u) {
+            const int pix = (u * NUM_PRODUCERS + ptid) >> 3;
+            const int py = pix / PW, px = pix - py * PW;
+            // row = halo pixel (128 B = 64 channels), 16-byte chunk c stored at c ^ (row & 7): the
+            // 128-byte swizzle of the K-major operand layout (tile bases are 1024-byte aligned).
+            // bf16 input: the thread's channels [8j, 8j+8) are chunk j.  fp32 input: channels
+            // [4j, 4j+4) are half (j & 1) of chunk j / 2 and [32+4j, ..) the same half of chunk 4 + j / 2,
+            // whose offset differs from the first by exactly 64 bytes (bit 2 of the chunk number).
+            soff[u] = IN_BF16 ? (uint32_t)(pix * 128 + ((j ^ (pix & 7)) << 4))
+                              : (uint32_t)(pix * 128 + (((j >> 1) ^ (pix & 7)) << 4) + (j & 1) * 8);
+            goff[u] = ((((py - 1) >> up) * a.Ws + ((px - 1) >> up)) * a.Cin) * ESZ;
+            const bool inner = py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
+            pyx[u] = (uint32_t)py | ((uint32_t)px << 8) | (inner ? 1u << 16 : 0u);
+        }
         Tracer tr; tr.init(ptid == 0 ? a.trace : nullptr, 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
-        Pos cur;
-        cur.t = sched.begin; cur.kc = 0; cur.slot = 0; cur.cnt = 1;
-        if (cur.t < sched.end) { cur.cnt = sched.count(cur.t); cur.tile = sched.get(cur.t, BN); }
-        while (cur.t < sched.end && ok) {
-            const bool second = cur.kc >= kchunks;
-            const bool in_bf16 = second ? false : IN_BF16;
-            const int c0 = (second ? cur.kc - kchunks : cur.kc) * 64;
-            const bool centre_only = second || a.ksize == 1;
-            tr.mark(1);
-            Raw8 raw[BATCH];
-            uint32_t vm = 0;
+        for (int t = sched.begin; t < sched.end && ok;) {
+            const int cnt = sched.count(t);
+            const Tile tile0 = sched.get(t, BN);
+            for (int kc = 0; kc < ktotal && ok; ++kc) {
+                const bool second = kc >= kchunks;
+                const int c0 = (second ? kc - kchunks : kc) * 64;
+                const bool centre_only = second || a.ksize == 1;
+                const bool pro = prologue && !second;
+                float sc[8], sh[8];
+                if (pro) {
+                    // channels of v[0..3] and v[4..7] (see load_raw); the tiles of an item lie in one frame
+                    const int ca = c0 + (IN_BF16 ? j * 8 : j * 4), cb = IN_BF16 ? ca + 4 : ca + 32;
+                    const float* ps = a.scale + (size_t)tile0.b * a.Cin;
+                    const float* pt = a.shift + (size_t)tile0.b * a.Cin;
+                    const float4 s0 = __ldg((const float4*)(ps + ca)), s1 = __ldg((const float4*)(ps + cb));
+                    const float4 t0 = __ldg((const float4*)(pt + ca)), t1 = __ldg((const float4*)(pt + cb));
+                    sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
+                    sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
+                    if (silu) {          // SiLU is evaluated as h + h*tanh(h) with h = v/2: the 1/2 folds into the affine map
 #pragma unroll
-            for (int u = 0; u < BATCH; ++u) {
-                const int pix = (u * NUM_PRODUCERS + ptid) >> 3;
-                const int py = pix / PW, px = pix - py * PW;
-                const int oy = cur.tile.ty0 + py - 1, ox = cur.tile.tx0 + px - 1;
-                bool v = oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
-                if (centre_only) v = v && py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
-                if (v) {
-                    vm |= 1u << u;
-                    if (second) load_raw(false, a.x2, (((size_t)cur.tile.b * a.H + oy) * a.W + ox) * a.Cin2, c0, j, raw[u]);
-                    else load_raw(IN_BF16, a.x, (((size_t)cur.tile.b * a.Hs + (oy >> up)) * a.Ws + (ox >> up)) * a.Cin, c0, j, raw[u]);
-                }
-            }
-            const bool pro = prologue && !second;
-            float sc[8], sh[8];
-            if (pro) {
-                // channels of v[0..3] and v[4..7] (see load_raw)
-                const int ca = c0 + (in_bf16 ? j * 8 : j * 4), cb = in_bf16 ? ca + 4 : ca + 32;
-                const float* ps = a.scale + (size_t)cur.tile.b * a.Cin;
-                const float* pt = a.shift + (size_t)cur.tile.b * a.Cin;
-                const float4 s0 = __ldg((const float4*)(ps + ca)), s1 = __ldg((const float4*)(ps + cb));
-                const float4 t0 = __ldg((const float4*)(pt + ca)), t1 = __ldg((const float4*)(pt + cb));
-                sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
-                sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
-            }
-            if (cur.slot == 0) {
-                ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
-                if (!ok) break;
-            }
-            tr.mark(2);
-            uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur.slot * A_TILE_BYTES;
-#pragma unroll
-            for (int u = 0; u < BATCH; ++u) {
-                uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
-                if (vm & (1u << u)) {
-                    float v[8];
-                    unpack_raw(in_bf16, raw[u], v);
-                    if (pro) {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
-                        if (silu) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) v[e] = silu_fast(v[e]);
-                        }
+                        for (int e = 0; e < 8; ++e) { sc[e] *= 0.5f; sh[e] *= 0.5f; }
                     }
-                    o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]);
                 }
-                // row = halo pixel (128 B = 64 channels), 16-byte chunk c stored at c ^ (row & 7): the
-                // 128-byte swizzle of the K-major operand layout (tile bases are 1024-byte aligned)
-                const int pix = (u * NUM_PRODUCERS + ptid) >> 3;
-                uint8_t* prow = dst_tile + pix * 128;
-                if (in_bf16) {
-                    *(uint4*)(prow + ((j ^ (pix & 7)) << 4)) = make_uint4(o0, o1, o2, o3);
-                } else {     // channels 4j..4j+3 -> chunk j/2, half j&1; channels 32+4j.. -> chunk 4 + j/2
-                    const int c = j >> 1, hb = (j & 1) * 8;
-                    *(uint2*)(prow + ((c ^ (pix & 7)) << 4) + hb) = make_uint2(o0, o1);
-                    *(uint2*)(prow + (((c + 4) ^ (pix & 7)) << 4) + hb) = make_uint2(o2, o3);
+#pragma unroll
+                for (int slot = 0; slot < PAIR; ++slot) {
+                    if (slot < cnt) {
+                        Tile tile = tile0;                   // the second tile of an item is the next one in its channel block
+                        if (slot == 1) {
+                            tile.tx0 += TILE_W;
+                            if (tile.tx0 >= sched.tiles_x * TILE_W) { tile.tx0 = 0; tile.ty0 += TILE_H; }
+                        }
+                        tr.mark(1);
+                        // which entries exist: all of them where the halo lies inside the image
+                        uint32_t vm = 7u;
+                        const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
+                        if (!interior || centre_only) {
+                            vm = 0u;
+#pragma unroll
+                            for (int u = 0; u < BATCH; ++u) {
+                                const int oy = tile.ty0 + (int)(pyx[u] & 0xffu) - 1, ox = tile.tx0 + (int)((pyx[u] >> 8) & 0xffu) - 1;
+                                bool v = oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
+                                if (centre_only) v = v && (pyx[u] >> 16) != 0u;
+                                vm |= (v ? 1u : 0u) << u;
+                            }
+                        }
+                        Raw8 raw[BATCH];
+                        if (!second) {
+                            const char* xb = (const char*)a.x
+                                + ((((size_t)tile.b * a.Hs + (tile.ty0 >> up)) * a.Ws + (tile.tx0 >> up)) * a.Cin + c0 + (IN_BF16 ? j * 8 : j * 4)) * ESZ;
+#pragma unroll
+                            for (int u = 0; u < BATCH; ++u)
+                                if (vm & (1u << u)) load_raw_at(IN_BF16, xb + goff[u], raw[u]);
+                        } else {             // fused shortcut: fp32 input at the output resolution, centre pixels only
+                            const char* xb = (const char*)a.x2 + ((((size_t)tile.b * a.H + tile.ty0) * a.W + tile.tx0) * a.Cin2 + c0 + j * 4) * 4;
+#pragma unroll
+                            for (int u = 0; u < BATCH; ++u)
+                                if (vm & (1u << u))
+                                    load_raw_at(false, xb + (((int)(pyx[u] & 0xffu) - 1) * a.W + ((int)((pyx[u] >> 8) & 0xffu) - 1)) * a.Cin2 * 4, raw[u]);
+                        }
+                        if (slot == 0) {
+                            ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
+                            if (!ok) break;
+                        }
+                        tr.mark(2);
+                        uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + slot * A_TILE_BYTES;
+                        const bool in_bf16 = IN_BF16 && !second;
+#pragma unroll
+                        for (int u = 0; u < BATCH; ++u) {
+                            uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
+                            if (vm & (1u << u)) {
+                                float v[8];
+                                unpack_raw(in_bf16, raw[u], v);
+                                if (pro) {
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
+                                    if (silu) {
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], tanh_fast(v[e]), v[e]);
+                                    }
+                                }
+                                o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]);
+                            }
+                            if (in_bf16) {
+                                *(uint4*)(dst_tile + soff[u]) = make_uint4(o0, o1, o2, o3);
+                            } else {
+                                uint32_t so = soff[u];
+                                if (IN_BF16) {               // fp32 second input of a kernel whose first input is bf16
+                                    const uint32_t pix = so >> 7;
+                                    so = pix * 128 + (((j >> 1) ^ (pix & 7)) << 4) + (j & 1) * 8;
+                                }
+                                *(uint2*)(dst_tile + so) = make_uint2(o0, o1);
+                                *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
+                            }
+                        }
+                        tr.mark(3);
+                    }
                 }
-            }
-            if (cur.slot == cur.cnt - 1) {
+                if (!ok) break;
                 fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[stage]));
                 if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
             }
-            tr.mark(3);
-            advance(cur);
+            t += cnt;
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------ epilogue
@@ -425,13 +461,20 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
             }
         }
-    } else if (warp == MMA_WARP) {
+    } else if (warp == MMA_WARP || (PAIR == 2 && warp == MMA_WARP2)) {
         // ------------------------------------------------ MMA issue
+        // Issuing one tcgen05.mma costs its thread about 50 cycles, and a wait plus a commit about
+        // 230 more, so one thread cannot feed eight N=128 MMAs per weight stage (513 tensor
+        // cycles).  Where an item is two tiles, each tile has its own issuing thread (in its own
+        // warp): both follow every barrier in lockstep and both arrive on the "empty"/"full"
+        // barriers they release, by tcgen05.commit when they issued MMAs and plainly when an odd
+        // tail item has no second tile.
         if (lane == 0) {
+            const int me = warp == MMA_WARP ? 0 : 1;          // the tile slot this thread issues for
             constexpr uint32_t idesc = make_idesc_bf16(128, BN);
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
-            const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)), b_lo0 = desc_lo(smem_u32(smem_b));
-            Tracer tr; tr.init(a.trace, 1);
+            const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)) + me * (A_TILE_BYTES >> 4), b_lo0 = desc_lo(smem_u32(smem_b));
+            Tracer tr; tr.init(me == 0 ? a.trace : nullptr, 1);
             tr.mark_at(40, t_entry);
             tr.mark(41);
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
@@ -439,13 +482,14 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             int n_item = 0;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int cnt = sched.count(t);
+                const bool active = me < cnt;
                 const int buf = n_item % NBUF;
                 tr.mark(20);
                 ok = mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 tr.mark(21);
-                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
+                const uint32_t td = tmem_base + (uint32_t)((buf * PAIR + me) * Cfg::ACC_COLS);
                 uint32_t acc = 0;                             // the first MMA of an item overwrites the accumulator
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
@@ -458,8 +502,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     // tap view: rows start (ky*PW + kx) pixels into the halo tile; eight-row groups are
                     // one tile row (PW pixels) apart.  The tensor core applies the 128-byte swizzle to the
                     // absolute shared-memory address, so any 128-byte-aligned start works (base_offset 0).
-                    const uint32_t a_chunk = a_lo0 + as * (A_STAGE_BYTES >> 4);
-                    uint32_t tap_off = centre ? (PW + 1) * 8 : 0;              // (ky*PW + kx) * 128 B >> 4
+                    uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (centre ? (PW + 1) * 8 : 0);   // + (ky*PW + kx) * 128 B >> 4
                     int kx = 0;
                     for (int tap = 0; tap < ntap; ++tap) {
                         tr.mark_fine(25);
@@ -468,27 +511,29 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         tc_fence_after();
                         tr.mark_fine(24);
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
-                        uint32_t a_lo = a_chunk + tap_off;
-                        uint32_t td = tmem_d;
-                        for (int slot = 0; slot < cnt; ++slot) {
+                        if (active) {
                             umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
                             umma_bf16_split(td, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc, 1u);
                             umma_bf16_split(td, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc, 1u);
                             umma_bf16_split(td, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc, 1u);
-                            a_lo += A_TILE_BYTES >> 4;
-                            td += Cfg::ACC_COLS;
                         }
                         acc = 1u;
-                        // tcgen05.commit is served at a limited rate (about one per 700 cycles), so weight
-                        // stages are handed back B_GROUP at a time
-                        if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                        // weight stages are handed back B_GROUP at a time (fewer commits on the issuing thread)
+                        if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) {
+                            if (active) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                            else mbar_arrive(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                        }
                         if (++bs == Cfg::B_STAGES) { bs = 0; bph ^= 1; }
-                        if (++kx == 3) { kx = 0; tap_off += (PW - 2) * 8; } else tap_off += 8;
+                        if (++kx == 3) { kx = 0; a_lo += (PW - 2) * 8; } else a_lo += 8;
                     }
-                    umma_commit(smem_u32(&bars->a_empty[as]));
+                    if (active) umma_commit(smem_u32(&bars->a_empty[as]));
+                    else mbar_arrive(smem_u32(&bars->a_empty[as]));
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
-                if (ok) umma_commit(smem_u32(&bars->acc_full[buf]));
+                if (ok) {
+                    if (active) umma_commit(smem_u32(&bars->acc_full[buf]));
+                    else mbar_arrive(smem_u32(&bars->acc_full[buf]));
+                }
                 t += cnt;
             }
         }

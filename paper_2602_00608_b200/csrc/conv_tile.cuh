@@ -22,9 +22,10 @@ static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the ha
 // MMA-issuing thread no priority: measured, fifteen warps of dense arithmetic stretch its
 // wait / 4 x MMA / commit sequence from 513 to about 1800 cycles, while the same warps kept off its
 // sub-partition cost nothing.  So sub-partition 0 carries only the MMA warp, the TMA warp and one
-// epilogue warp (warps 8, 12 and 20 idle until the end), and the fifteen producer warps are the
+// epilogue warp (warp 8 is the second MMA warp of two-tile items; warps 12 and 20 idle until the end), and the fifteen producer warps are the
 // warps with warp % 4 != 0 outside the epilogue: five per remaining sub-partition.
 constexpr int MMA_WARP = 0;
+constexpr int MMA_WARP2 = 8;                                        // second issuing thread where an item is two tiles
 constexpr int TMA_WARP = 4;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
 constexpr int NUM_THREADS = 24 * 32;
@@ -44,6 +45,16 @@ __device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix
     } else {
         const float* p = (const float*)x + pix_off + c0 + j * 4;
         const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 32));
+        r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
+        r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
+    }
+}
+// the same loads from the address of the thread's first channel
+__device__ __forceinline__ void load_raw_at(bool is_bf16, const char* p, Raw8& r) {
+    if (is_bf16) {
+        r.lo = __ldg((const uint4*)p);
+    } else {
+        const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 128));
         r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
         r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
     }

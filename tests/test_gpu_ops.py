@@ -199,9 +199,12 @@ def test_conv_tc_matches_oracle(env, case):
     # output adds one more rounding of the result
     tol = 4e-3 if case["out_bf16"] else 2.5e-3
     assert rel_l2(got, want) <= tol
-    # and the two GPU implementations agree far more closely than either does with fp32 math
+    # and the two GPU implementations agree far more closely than either does with fp32 math.
+    # With SiLU in the prologue the tensor-core kernel uses the hardware tanh (relative error
+    # 2^-11, an eighth of a bf16 rounding step), which moves a small fraction of the operands
+    # across a bf16 rounding boundary; without it the operands are bitwise the same.
     got2, _ = _conv_case(env, seed=41, impl=vd.VD_IMPL_SIMT, bf16_ops=True, **case)
-    assert rel_l2(got, got2) <= (4e-3 if case["out_bf16"] else 2e-5)
+    assert rel_l2(got, got2) <= (4e-3 if case["out_bf16"] else (2e-4 if case["silu"] else 2e-5))
 
 
 def test_conv_tc_real_layer_shape_sampled(env):
