@@ -463,18 +463,20 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         }
     } else if (warp == MMA_WARP || (PAIR == 2 && warp == MMA_WARP2)) {
         // ------------------------------------------------ MMA issue
-        // Issuing one tcgen05.mma costs its thread about 50 cycles, and a wait plus a commit about
-        // 230 more, so one thread cannot feed eight N=128 MMAs per weight stage (513 tensor
-        // cycles).  Where an item is two tiles, each tile has its own issuing thread (in its own
-        // warp): both follow every barrier in lockstep and both arrive on the "empty"/"full"
-        // barriers they release, by tcgen05.commit when they issued MMAs and plainly when an odd
-        // tail item has no second tile.
-        if (lane == 0) {
-            const int me = warp == MMA_WARP ? 0 : 1;          // the tile slot this thread issues for
+        // The whole warp runs the loop and one elected lane issues: in warp-uniform code the
+        // compiler keeps descriptors and counters in uniform registers, and the issue sequence of
+        // wait / 4 x tcgen05.mma / commit costs about 300 cycles instead of about 480 from a
+        // single-lane branch (measured), which a tap's 513 tensor cycles then hide.  Where an item
+        // is two tiles, each tile has its own issuing warp: both follow every barrier in lockstep
+        // and both arrive on the "empty"/"full" barriers they release, by tcgen05.commit when they
+        // issued MMAs and plainly when an odd tail item has no second tile.
+        {
+            const int me = warp == MMA_WARP ? 0 : 1;          // the tile slot this warp issues for
+            const bool leader = elect_one() != 0u;
             constexpr uint32_t idesc = make_idesc_bf16(128, BN);
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
             const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)) + me * (A_TILE_BYTES >> 4), b_lo0 = desc_lo(smem_u32(smem_b));
-            Tracer tr; tr.init(me == 0 ? a.trace : nullptr, 1);
+            Tracer tr; tr.init((me == 0 && lane == 0) ? a.trace : nullptr, 1);
             tr.mark_at(40, t_entry);
             tr.mark(41);
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
@@ -485,7 +487,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const bool active = me < cnt;
                 const int buf = n_item % NBUF;
                 tr.mark(20);
-                ok = mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 tr.mark(21);
@@ -495,7 +497,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
                     const int ntap = centre ? 1 : 9;
                     tr.mark(22);
-                    ok = mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                     tr.mark(23);
@@ -506,34 +508,41 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     int kx = 0;
                     for (int tap = 0; tap < ntap; ++tap) {
                         tr.mark_fine(25);
-                        ok = mbar_wait(smem_u32(&bars->b_full[bs]), bph, abort_flag);
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->b_full[bs]), bph, abort_flag));
                         if (!ok) break;
                         tc_fence_after();
                         tr.mark_fine(24);
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
-                        if (active) {
-                            umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
-                            umma_bf16_split(td, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc, 1u);
-                            umma_bf16_split(td, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc, 1u);
-                            umma_bf16_split(td, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc, 1u);
+                        if (leader) {
+                            if (active) {
+                                umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
+                                umma_bf16_split(td, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc, 1u);
+                                umma_bf16_split(td, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc, 1u);
+                                umma_bf16_split(td, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc, 1u);
+                            }
+                            // weight stages are handed back B_GROUP at a time (fewer commits)
+                            if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) {
+                                if (active) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                                else mbar_arrive(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                            }
                         }
+                        __syncwarp();
                         acc = 1u;
-                        // weight stages are handed back B_GROUP at a time (fewer commits on the issuing thread)
-                        if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) {
-                            if (active) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
-                            else mbar_arrive(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
-                        }
                         if (++bs == Cfg::B_STAGES) { bs = 0; bph ^= 1; }
                         if (++kx == 3) { kx = 0; a_lo += (PW - 2) * 8; } else a_lo += 8;
                     }
-                    if (active) umma_commit(smem_u32(&bars->a_empty[as]));
-                    else mbar_arrive(smem_u32(&bars->a_empty[as]));
+                    if (leader) {
+                        if (active) umma_commit(smem_u32(&bars->a_empty[as]));
+                        else mbar_arrive(smem_u32(&bars->a_empty[as]));
+                    }
+                    __syncwarp();
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
-                if (ok) {
+                if (ok && leader) {
                     if (active) umma_commit(smem_u32(&bars->acc_full[buf]));
                     else mbar_arrive(smem_u32(&bars->acc_full[buf]));
                 }
+                __syncwarp();
                 t += cnt;
             }
         }

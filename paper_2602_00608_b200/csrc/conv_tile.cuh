@@ -51,6 +51,9 @@ __device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix
 }
 // the same loads from the address of the thread's first channel
 __device__ __forceinline__ void load_raw_at(bool is_bf16, const char* p, Raw8& r) {
+#ifdef VD_ABL_NOLOAD      // timing study: no global loads (results are wrong)
+    r.lo = make_uint4((uint32_t)(uintptr_t)p, 2u, 3u, 4u); r.hi = r.lo; return;
+#endif
     if (is_bf16) {
         r.lo = __ldg((const uint4*)p);
     } else {
