@@ -422,6 +422,68 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
             tr.mark(12);
         }
+    } else if (warp == PREFETCH_WARP) {
+        // ------------------------------------------------ input prefetch into L2
+        // The activations of the large layers do not fit the L2 cache, and a producer thread can
+        // keep only one unit of loads in flight in its registers, which does not cover the latency
+        // of device memory.  This warp follows the producers' progress on the operand barriers and
+        // asks L2, PF_AHEAD chunks ahead of them, for the 64-channel pixel records the chunk's
+        // tiles will read (one prefetch per 128-byte line; bulk prefetches of such small ranges
+        // would crowd the copy engine that also brings the weights).  It is best effort: a wait that
+        // runs out ends the role quietly.
+        griddep_wait();
+        constexpr int PF_AHEAD = 2;
+        const int esz = IN_BF16 ? 2 : 4;
+        const int h = a.ksize == 3 ? 1 : 0;
+        const int up = a.upsample ? 1 : 0;
+        int waited = 0;                                      // chunks of the CTA whose completion has been observed
+        int q = 0;                                           // chunk being prefetched (counted over the CTA's work)
+        bool ok = true;
+        for (int t = sched.begin; t < sched.end && ok;) {
+            const int cnt = sched.count(t);
+            Tile tl[PAIR];
+#pragma unroll
+            for (int sl = 0; sl < PAIR; ++sl) tl[sl] = sched.get(sl < cnt ? t + sl : t, BN);
+            for (int kc = 0; kc < ktotal && ok; ++kc, ++q) {
+                while (waited < q - PF_AHEAD + 1 && ok) {   // stay at most PF_AHEAD chunks ahead of the producers
+                    const uint32_t bar = smem_u32(&bars->a_full[waited % Cfg::A_STAGES]);
+                    const uint32_t par = (uint32_t)(waited / Cfg::A_STAGES) & 1u;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(bar, par)) {
+                        __nanosleep(200);
+                        if (*abort_flag || clock64() - t0 > 400000) { ok = false; break; }
+                    }
+                    ++waited;
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const bool second = kc >= kchunks;
+#pragma unroll
+                for (int sl = 0; sl < PAIR; ++sl) {
+                    if (sl >= cnt) continue;
+                    if (!second) {
+                        const int y0 = max(tl[sl].ty0 - h, 0) >> up, y1 = (min(tl[sl].ty0 + TILE_H + h, a.H) - 1) >> up;
+                        const int x0 = max(tl[sl].tx0 - h, 0) >> up, x1 = (min(tl[sl].tx0 + TILE_W + h, a.W) - 1) >> up;
+                        const int rw = x1 - x0 + 1, n = rw * (y1 - y0 + 1);
+                        const char* base = (const char*)a.x + (((size_t)tl[sl].b * a.Hs * a.Ws) * a.Cin + kc * 64) * esz;
+                        const int lpp = IN_BF16 ? 1 : 2;            // 128-byte lines per pixel record
+                        for (int i = lane; i < n * lpp; i += 32) {
+                            const int px = IN_BF16 ? i : i >> 1, ln = IN_BF16 ? 0 : i & 1;
+                            const int ry = px / rw, rx = px - ry * rw;
+                            prefetch_l2(base + ((size_t)(y0 + ry) * a.Ws + (x0 + rx)) * a.Cin * esz + ln * 128);
+                        }
+                    } else {
+                        const int rw = min(tl[sl].tx0 + TILE_W, a.W) - tl[sl].tx0, n = rw * (min(tl[sl].ty0 + TILE_H, a.H) - tl[sl].ty0);
+                        const char* base = (const char*)a.x2 + (((size_t)tl[sl].b * a.H * a.W) * a.Cin2 + (kc - kchunks) * 64) * 4;
+                        for (int i = lane; i < n * 2; i += 32) {
+                            const int px = i >> 1, ry = px / rw, rx = px - ry * rw;
+                            prefetch_l2(base + ((size_t)(tl[sl].ty0 + ry) * a.W + (tl[sl].tx0 + rx)) * a.Cin2 * 4 + (i & 1) * 128);
+                        }
+                    }
+                }
+            }
+            t += cnt;
+        }
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
         if (lane == 0) {

@@ -49,6 +49,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
+// L2 prefetch of the 128-byte line that holds p
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 // one lane of a converged warp (the same one every time)
 __device__ __forceinline__ uint32_t elect_one() {
     uint32_t p;
