@@ -230,49 +230,60 @@ attn_tc_kernel(const AttnTcParams a, const __grid_constant__ CUtensorMap tm_q, c
         }
     } else {
         // ------------------------------------------------------------ MMA issue
-        if (lane == 0) {
+        // The whole warp runs the loop and one elected lane issues: warp-uniform code keeps the
+        // descriptors in uniform registers, which makes the wait / 4 x MMA / commit sequence of a
+        // 64-channel chunk cheaper than the 256 tensor cycles it feeds.
+        {
+            const bool leader = elect_one() != 0u;
             constexpr uint32_t idesc_s = make_idesc_bf16(128, BKV);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, DV);
+            const uint32_t hi = desc_hi(1024, 2);
             uint32_t qst = 0, qph = 0, vst = 0, vph = 0;
             bool ok = true;
             auto issue_qk = [&](int j) {
                 const int buf = j & 1;
-                ok = mbar_wait(smem_u32(&bars->s_free[buf]), ((j >> 1) & 1) ^ 1, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_free[buf]), ((j >> 1) & 1) ^ 1, abort_flag));
                 if (!ok) return;
                 tc_fence_after();
                 for (int dc = 0; dc < dchunks; ++dc) {
-                    ok = mbar_wait(smem_u32(&bars->qk_full[qst]), qph, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->qk_full[qst]), qph, abort_flag));
                     if (!ok) return;
                     tc_fence_after();
-                    const uint32_t qa = smem_u32(smem_qk + qst * QK_STAGE_BYTES);
-                    const uint32_t ka = qa + BQ * DCHUNK * 2;
+                    const uint32_t qa = desc_lo(smem_u32(smem_qk + qst * QK_STAGE_BYTES));
+                    const uint32_t ka = qa + ((BQ * DCHUNK * 2) >> 4);
+                    if (leader) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem + (uint32_t)(buf * 128), make_smem_desc(qa + k * 32, 16, 1024, 2),
-                                  make_smem_desc(ka + k * 32, 16, 1024, 2), idesc_s, (dc | k) != 0);
-                    umma_commit(smem_u32(&bars->qk_empty[qst]));
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16_split(tmem + (uint32_t)(buf * 128), qa + k * 2, hi, ka + k * 2, hi, idesc_s, (dc | k) != 0 ? 1u : 0u);
+                        umma_commit(smem_u32(&bars->qk_empty[qst]));
+                    }
+                    __syncwarp();
                     if (++qst == QK_STAGES) { qst = 0; qph ^= 1; }
                 }
-                umma_commit(smem_u32(&bars->s_full[buf]));
+                if (leader) umma_commit(smem_u32(&bars->s_full[buf]));
+                __syncwarp();
             };
             auto issue_pv = [&](int j) {
-                ok = mbar_wait(smem_u32(&bars->p_full), j & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full), j & 1, abort_flag));
                 if (!ok) return;
                 tc_fence_after();
                 for (int h = 0; h < 2; ++h) {
-                    ok = mbar_wait(smem_u32(&bars->v_full[vst]), vph, abort_flag);
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->v_full[vst]), vph, abort_flag));
                     if (!ok) return;
                     tc_fence_after();
-                    const uint32_t pa = smem_u32(smem_p + h * (BQ * 128));
-                    const uint32_t va = smem_u32(smem_v + vst * V_STAGE_BYTES);
+                    const uint32_t pa = desc_lo(smem_u32(smem_p + h * (BQ * 128)));
+                    const uint32_t va = desc_lo(smem_u32(smem_v + vst * V_STAGE_BYTES));
+                    if (leader) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem_o, make_smem_desc(pa + k * 32, 16, 1024, 2), make_smem_desc(va + k * 32, 16, 1024, 2),
-                                  idesc_o, (j | h | k) != 0);
-                    umma_commit(smem_u32(&bars->v_empty[vst]));
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16_split(tmem_o, pa + k * 2, hi, va + k * 2, hi, idesc_o, (j | h | k) != 0 ? 1u : 0u);
+                        umma_commit(smem_u32(&bars->v_empty[vst]));
+                    }
+                    __syncwarp();
                     if (++vst == V_STAGES) { vst = 0; vph ^= 1; }
                 }
-                umma_commit(smem_u32(&bars->pv_done));
+                if (leader) umma_commit(smem_u32(&bars->pv_done));
+                __syncwarp();
             };
             issue_qk(0);
             for (int j = 0; j < ntiles && ok; ++j) {
