@@ -84,18 +84,32 @@ def contract_roofline_us(steps, peaks, batch, stream_bytes=2):
 
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,"
+             "timestamp")
 
     def __init__(self, gpu_index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "50", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
-    def stop(self):
+    def wait_for_samples(self, n: int, timeout_s: float = 5.0):
+        """Blocks until nvidia-smi has written n lines (it takes a moment to start)."""
+        t0 = time.time()
+        while self.p is not None and time.time() - t0 < timeout_s:
+            try:
+                if sum(1 for _ in open(self.f.name)) >= n:
+                    return
+            except OSError:
+                pass
+            time.sleep(0.02)
+
+    def stop(self, t_begin: float = None, t_end: float = None):
+        """Summary of the samples taken between the two time.time() stamps (all samples if none given)."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
             return out
@@ -109,9 +123,12 @@ class ClockSampler:
         sm, mx, pw, reasons = [], [], [], set()
         for line in self.f.read().splitlines():
             c = [x.strip() for x in line.split(",")]
-            if len(c) < 9:
+            if len(c) < 10:
                 continue
             try:
+                ts = datetime.datetime.strptime(c[9], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
+                    continue
                 sm.append(float(c[1])); mx.append(float(c[2])); pw.append(float(c[3]))
             except ValueError:
                 continue
@@ -124,6 +141,12 @@ class ClockSampler:
             out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
                        power_w_max=max(pw))
         return out
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the launches of one decode)
+# of the dominant kernel, from one ncu capture of this program on the named workload; the capture and
+# its command are summarised under profiles/.  Other workloads have no capture: null.
+NCU_DRAM_BYTES_PER_LAUNCH = {("sdvae-bf16-720x480", "conv_tc"): 137.6e6}
 
 
 def time_oracle(wl, crop, steps, warmup):
@@ -162,8 +185,8 @@ def run_reference(args, wl, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=3, help="workload index (3 = 720x480 headline)")
     ap.add_argument("--impl", default="vd", choices=["vd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -216,19 +239,32 @@ def main():
         return float(t.item())
 
     # ---- device-resident timing
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(args.warmup):
         dec.decode(z, frames)
+    if sampler:                      # nvidia-smi needs a moment to start: keep the GPU under the same load meanwhile
+        t_w = time.time()
+        while time.time() - t_w < 3.0:
+            for _ in range(10):
+                dec.decode(z, frames)
+            torch.cuda.synchronize()
+            try:
+                if sum(1 for _ in open(sampler.f.name)) >= 2:
+                    break
+            except OSError:
+                break
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_begin = time.time()
     e0.record(stream)
     for _ in range(args.steps):
         dec.decode(z, frames)
     e1.record(stream)
     barrier()
+    t_end = time.time()
     ms_total = max_over_ranks(e0.elapsed_time(e1))
     dec.check_status()
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop(t_begin, t_end) if sampler else None
     ms_step = ms_total / args.steps
     fps = world * wl.batch * args.steps / (ms_total * 1e-3)
 
@@ -280,7 +316,8 @@ def main():
     if d["flops"] > 0:
         roof = {"kernel": dom, "bound": "tensor", "achieved": d["flops"] / (d["ms"] * 1e-3) / 1e12, "peak": peak_tf,
                 "unit": "TFLOP/s", "peak_source": f"{peaks['source']} (sustained: kernel timed inside a long step)",
-                "traffic": None, "launches_per_step": d["launches"], "ms_per_step": d["ms"]}
+                "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dom)), "traffic_unit": "bytes per launch (ncu, cold cache)",
+                "launches_per_step": d["launches"], "ms_per_step": d["ms"]}
     else:
         roof = {"kernel": dom, "bound": "hbm", "achieved": d["bytes"] / (d["ms"] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "peak_source": peaks["source"], "traffic": None, "launches_per_step": d["launches"],
