@@ -50,18 +50,20 @@ __device__ __forceinline__ void load_raw(bool is_bf16, const void* x, size_t pix
         r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
     }
 }
-// the same loads from the address of the thread's first channel
+// the same loads from the address of the thread's first channel.  The activations are streamed
+// (no reuse within the SM): they bypass L1 allocation, which leaves the small L1 that remains beside
+// the shared-memory tiles to the data that is reused.
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
 __device__ __forceinline__ void load_raw_at(bool is_bf16, const char* p, Raw8& r) {
 #ifdef VD_ABL_NOLOAD      // timing study: no global loads (results are wrong)
     r.lo = make_uint4((uint32_t)(uintptr_t)p, 2u, 3u, 4u); r.hi = r.lo; return;
 #endif
-    if (is_bf16) {
-        r.lo = __ldg((const uint4*)p);
-    } else {
-        const float4 a = __ldg((const float4*)p), b = __ldg((const float4*)(p + 128));
-        r.lo = make_uint4(__float_as_uint(a.x), __float_as_uint(a.y), __float_as_uint(a.z), __float_as_uint(a.w));
-        r.hi = make_uint4(__float_as_uint(b.x), __float_as_uint(b.y), __float_as_uint(b.z), __float_as_uint(b.w));
-    }
+    r.lo = ldg_stream(p);
+    if (!is_bf16) r.hi = ldg_stream(p + 128);
 }
 __device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[8]) {
     if (is_bf16) {
