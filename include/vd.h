@@ -211,7 +211,9 @@ VD_API vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* 
 /* GroupNorm statistics of x (device NHWC [batch,h,w,c], dtype `dtype`) folded with the affine
  * parameters: scale[n,c] = gamma[c]*rstd[n,g], shift[n,c] = beta[c] - mean[n,g]*scale[n,c]
  * (biased variance, eps inside the root).  `scratch` is device memory of
- * vd_gn_scratch_bytes(batch, groups) bytes.  scale/shift are device fp32 [batch,c]. */
+ * vd_gn_scratch_bytes(batch, groups) bytes (chunk records, then one arrival counter per sample,
+ * which the call clears itself).  scale/shift are device fp32 [batch,c].  c <= 1024, c/groups a
+ * multiple of 4.  One kernel launch; results are bitwise reproducible and do not depend on batch. */
 VD_API size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups);
 VD_API vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w, int32_t c,
                                 int32_t groups, float eps, const float* gamma, const float* beta,
@@ -221,14 +223,15 @@ VD_API vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int
  * has no counterpart of this entry point; it exists for hosts where device allocation is not an
  * option at call time: frame loops that must not hit the allocator's implicit synchronisation,
  * plug-ins living inside another application's memory budget, code running in a host callback.
- * The chunk partials live in a 1 MiB array built into the library (held by every GPU that loads
- * it until the process exits).  Limits and rules:
+ * The chunk records and the arrival counters live in a 148 KiB array built into the library (held
+ * by every GPU that loads it until the process exits).  Limits and rules:
  *   - batch * groups <= 64, else VD_ERR_UNSUPPORTED (use vd_op_gn_stats);
  *   - no cudaMalloc/cudaFree or any allocating routine is called;
  *   - the first call on a device looks up the array's device address (with that device
  *     current); make that first call before starting any stream capture;
  *   - all calls on a device share the array: calls whose kernels may overlap on the GPU race.
- *     Nothing needs clearing between calls (each call writes every slot it later reads). */
+ *     The records need no clearing between calls (each call writes every record it later
+ *     reads); the arrival counters are cleared by an asynchronous memset at the start of a call. */
 VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w,
                                        int32_t c, int32_t groups, float eps, const float* gamma,
                                        const float* beta, float* scale, float* shift, void* cuda_stream);
