@@ -231,12 +231,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    from paper_2602_00608_b200 import replicas
+
     def max_over_ranks(v: float) -> float:
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(v, world, dev)
 
     # ---- device-resident timing
     sampler = ClockSampler(local_rank) if rank == 0 else None
@@ -266,7 +264,7 @@ def main():
     dec.check_status()
     clocks = sampler.stop(t_begin, t_end) if sampler else None
     ms_step = ms_total / args.steps
-    fps = world * wl.batch * args.steps / (ms_total * 1e-3)
+    fps = replicas.whole_job_rate(world, wl.batch, args.steps, ms_total)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
     zh = torch.from_numpy(z_np).to(dec.dtype).pin_memory()
@@ -280,7 +278,7 @@ def main():
     e1.record(stream)
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
-    e2e = {"value": world * wl.batch / (e2e_ms * 1e-3), "unit": "frames/s",
+    e2e = {"value": replicas.whole_job_rate(world, wl.batch, 1, e2e_ms), "unit": "frames/s",
            "h2d_bytes_per_step": zh.numel() * zh.element_size(), "d2h_bytes_per_step": fh.numel() * fh.element_size(),
            "ms_per_step": e2e_ms}
 
