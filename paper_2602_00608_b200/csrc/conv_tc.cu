@@ -50,12 +50,22 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
 // item is two 16x8-pixel tiles whose MMAs consume every weight stage together, which halves the
 // weight traffic through shared memory and the bytes the TMA pipeline must keep in flight.
-template <int BN> struct TileCfg {
-    static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item
-    static constexpr int B_STAGE_BYTES = BN * 128;                   // BN rows x 64 bf16
-    static constexpr int B_STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+//
+// CG = 2 (BN = 256 only): a cluster of two CTAs on neighbouring SMs issues every MMA as one
+// tcgen05.mma.cta_group::2 of M = 256 (one tile per CTA) x N = 256.  Each CTA stages only its half of
+// every weight tile (128 rows) and the tensor cores of the pair read both halves, so the weight bytes
+// each SM pulls from L2 are halved; the one-CTA kernel is bound there by that traffic (32 KB per 513
+// tensor cycles and SM).  The MMA warp is active in the leader CTA (cluster rank 0) only.  Barriers
+// that gate the MMAs live in the leader: the peer's producers and weight loads signal the leader's
+// "full" barriers across the cluster, its epilogue the leader's "accumulator free" barrier, and the
+// leader's tcgen05.commit multicasts to the "empty" / "accumulator ready" barriers of both CTAs.
+template <int BN, int CG = 1> struct TileCfg {
+    static_assert(CG == 1 || BN == 256, "the two-CTA form exists for 256-channel blocks only");
+    static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
+    static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
+    static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 6 : 8));
     static constexpr int B_GROUP = 2;                                // weight stages handed back per tcgen05.commit
-    static constexpr int A_STAGES = 2;
+    static constexpr int A_STAGES = CG == 2 ? 3 : 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
@@ -78,9 +88,13 @@ struct Bars {                    // lives in shared memory
 // Tiles are numbered (frame, channel block, tile row, tile column), column fastest.  Every CTA
 // owns a contiguous, balanced range of tile numbers and walks it in items of `pair` tiles (one
 // when the range or the channel block ends).
+//
+// Two-CTA form: the range belongs to the cluster, an item is up to two tiles of one channel block,
+// and CTA `rank` of the pair takes tile t + rank (the peer has none in an odd tail item).
 struct Sched {
     int tiles_x, tiles, nblk, total;
     int begin, end, pair;
+    int cg, rank;
     __device__ __forceinline__ Tile get(int t, int bn) const {
         Tile r;
         const int blk = t / tiles;               // frame * nblk + channel block
@@ -93,17 +107,68 @@ struct Sched {
     }
     // number of tiles of the item that starts at tile t
     __device__ __forceinline__ int count(int t) const {
-        return (pair == 2 && t + 1 < end && (t + 1) / tiles == t / tiles) ? 2 : 1;
+        return ((pair == 2 || cg == 2) && t + 1 < end && (t + 1) / tiles == t / tiles) ? 2 : 1;
     }
+    // of those, the tiles this CTA works on, and the s-th of them
+    __device__ __forceinline__ int mine(int n) const { return cg == 2 ? (rank < n ? 1 : 0) : n; }
+    __device__ __forceinline__ int index(int t, int s) const { return cg == 2 ? t + rank : t + s; }
 };
+
+// ---- cluster / cta_group::2 PTX
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta) {     // shared::cta -> shared::cluster of `cta`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(cta));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// tile load into this CTA's shared memory whose completion is reported to a barrier of the leader CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, int x, int y, uint32_t leader_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(leader_bar) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16_split(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                 uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %6, 0;\n"
+        "mov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
 
 // OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC (both through shared memory and TMA stores),
 //           2 = NCHW frame written directly (dtype from a.out_dtype)
-template <int BN, bool IN_BF16, int OUT_MODE>
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, unsigned int* status) {
-    using Cfg = TileCfg<BN>;
+    using Cfg = TileCfg<BN, CG>;
     constexpr int NBUF = Cfg::NBUF, PAIR = Cfg::PAIR, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -126,22 +191,38 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     sched.tiles = sched.tiles_x * ((a.H + TILE_H - 1) / TILE_H);
     sched.nblk = cout_pad / BN;
     sched.total = sched.tiles * sched.nblk * a.B;
-    sched.begin = (int)(((long long)sched.total * blockIdx.x) / gridDim.x);
-    sched.end = (int)(((long long)sched.total * (blockIdx.x + 1)) / gridDim.x);
+    // work is divided among the CTAs (CG = 1) or among the clusters of two (CG = 2)
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;  // 0 = leader (issues the MMAs), 1 = peer
+    const int nworkers = (int)gridDim.x / CG, worker = (int)blockIdx.x / CG;
+    sched.begin = (int)(((long long)sched.total * worker) / nworkers);
+    sched.end = (int)(((long long)sched.total * (worker + 1)) / nworkers);
     sched.pair = PAIR;
+    sched.cg = CG;
+    sched.rank = (int)rank;
 
     if (tid == 0) {
-        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), PAIR); }
-        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), 1); mbar_init(smem_u32(&bars->b_empty[i]), PAIR); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), PAIR); mbar_init(smem_u32(&bars->acc_empty[i]), 4); }
+        // CG = 2: the leader's "full" barriers collect the arrivals of both CTAs; commits are multicast
+        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), CG * NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), PAIR); }
+        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), CG); mbar_init(smem_u32(&bars->b_empty[i]), PAIR); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), PAIR); mbar_init(smem_u32(&bars->acc_empty[i]), 4 * CG); }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
     }
-    if (warp == MMA_WARP) tmem_alloc(smem_u32(&bars->tmem_base), (uint32_t)Cfg::TMEM_COLS);
+    if (warp == MMA_WARP) {
+        if (CG == 2) tmem_alloc2(smem_u32(&bars->tmem_base), (uint32_t)Cfg::TMEM_COLS);
+        else tmem_alloc(smem_u32(&bars->tmem_base), (uint32_t)Cfg::TMEM_COLS);
+    }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                         // both CTAs' barriers exist before anyone signals across
     tc_fence_after();
+    // addresses, in the leader CTA, of the barriers that both CTAs signal
+    auto leader_bar = [&](uint64_t* b) -> uint32_t { return CG == 2 ? map_to_cta(smem_u32(b), 0) : smem_u32(b); };
+    auto arrive_leader = [&](uint64_t* b) {
+        if (CG == 2) mbar_arrive_cluster(map_to_cta(smem_u32(b), 0));
+        else mbar_arrive(smem_u32(b));
+    };
     const uint32_t tmem_base = bars->tmem_base;
     // The kernel after this one may set itself up from here on.  Of this kernel, only the roles
     // that touch activations wait for the kernel before it; weights (TMA warp) and the MMA issue
@@ -184,8 +265,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         for (int t = sched.begin; t < sched.end && ok;) {
-            const int cnt = sched.count(t);
-            const Tile tile0 = sched.get(t, BN);
+            const int n = sched.count(t);
+            const int cnt = sched.mine(n);                   // 0: the peer of a two-CTA pair in an odd tail item
+            const Tile tile0 = sched.get(cnt > 0 ? sched.index(t, 0) : t, BN);
             for (int kc = 0; kc < ktotal && ok; ++kc) {
                 const bool second = kc >= kchunks;
                 const int c0 = (second ? kc - kchunks : kc) * 64;
@@ -208,7 +290,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
 #pragma unroll
                 for (int slot = 0; slot < PAIR; ++slot) {
-                    if (slot < cnt) {
+                    if (slot < max(cnt, 1)) {
+                        const bool have = slot < cnt;        // without a tile the CTA still follows the barriers
                         Tile tile = tile0;                   // the second tile of an item is the next one in its channel block
                         if (slot == 1) {
                             tile.tx0 += TILE_W;
@@ -228,6 +311,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 vm |= (v ? 1u : 0u) << u;
                             }
                         }
+                        if (!have) vm = 0u;
                         Raw8 raw[BATCH];
                         if (!second) {
                             const char* xb = (const char*)a.x
@@ -251,6 +335,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const bool in_bf16 = IN_BF16 && !second;
 #pragma unroll
                         for (int u = 0; u < BATCH; ++u) {
+                            if (!have) break;
                             uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
                             if (vm & (1u << u)) {
                                 float v[8];
@@ -283,10 +368,10 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 if (!ok) break;
                 fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[stage]));
+                if (lane == 0) arrive_leader(&bars->a_full[stage]);
                 if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
             }
-            t += cnt;
+            t += n;
         }
     } else if (warp >= EPI_WARP0 && warp < EPI_WARP0 + 4) {
         // ------------------------------------------------ epilogue
@@ -343,16 +428,22 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
             int bias_n0 = -1;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
-                const int cnt = sched.count(t);
+                const int n = sched.count(t);
+                const int cnt = sched.mine(n);
                 const int buf = n_item % NBUF;
                 tr.mark(10);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 tr.mark(11);
+                if (cnt == 0) {                              // nothing of this CTA in the accumulators: hand them back at once
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) arrive_leader(&bars->acc_empty[buf]);
+                }
 #pragma unroll 1
                 for (int slot = 0; slot < cnt; ++slot) {
-                    const Tile tl = sched.get(t + slot, BN);
+                    const Tile tl = sched.get(sched.index(t, slot), BN);
                     if (tl.n0 != bias_n0) {                   // (re)load bias (+ shortcut bias) of this channel block
                         __syncwarp();
                         for (int i = lane; i < BN; i += 32)
@@ -402,7 +493,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         } else if (last_tile) {                          // accumulators fully read: hand them back
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                            if (lane == 0) arrive_leader(&bars->acc_empty[buf]);
                         }
                         if (h == PPS - 1) {
                             fence_proxy_async_smem();
@@ -417,7 +508,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     }
                     n_slice += NP / PPS;
                 }
-                t += cnt;
+                t += n;
             }
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
             tr.mark(12);
@@ -439,14 +530,18 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         int waited = 0;                                      // chunks of the CTA whose completion has been observed
         int q = 0;                                           // chunk being prefetched (counted over the CTA's work)
         bool ok = true;
+        // progress is read from the operand "full" barriers; in the two-CTA form those live in the leader
+        // only, so there it is read from the "empty" barriers (chunks consumed), A_STAGES chunks later
+        constexpr int PF_LEAD = CG == 2 ? PF_AHEAD + Cfg::A_STAGES : PF_AHEAD;
         for (int t = sched.begin; t < sched.end && ok;) {
-            const int cnt = sched.count(t);
+            const int n = sched.count(t);
+            const int cnt = sched.mine(n);
             Tile tl[PAIR];
 #pragma unroll
-            for (int sl = 0; sl < PAIR; ++sl) tl[sl] = sched.get(sl < cnt ? t + sl : t, BN);
+            for (int sl = 0; sl < PAIR; ++sl) tl[sl] = sched.get(sl < cnt ? sched.index(t, sl) : t, BN);
             for (int kc = 0; kc < ktotal && ok; ++kc, ++q) {
-                while (waited < q - PF_AHEAD + 1 && ok) {   // stay at most PF_AHEAD chunks ahead of the producers
-                    const uint32_t bar = smem_u32(&bars->a_full[waited % Cfg::A_STAGES]);
+                while (waited < q - PF_LEAD + 1 && ok) {    // stay at most PF_LEAD chunks ahead
+                    const uint32_t bar = smem_u32(CG == 2 ? &bars->a_empty[waited % Cfg::A_STAGES] : &bars->a_full[waited % Cfg::A_STAGES]);
                     const uint32_t par = (uint32_t)(waited / Cfg::A_STAGES) & 1u;
                     const long long t0 = clock64();
                     while (!mbar_try_wait(bar, par)) {
@@ -482,7 +577,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     }
                 }
             }
-            t += cnt;
+            t += n;
         }
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
@@ -503,10 +598,19 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             if (!ok) break;
                             tr.mark(31);
                         }
-                        const uint32_t full = smem_u32(&bars->b_full[stage]);
-                        mbar_arrive_expect_tx(full, Cfg::B_STAGE_BYTES);
-                        if (second) tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap2, (kc - kchunks) * 64, tl.n0, full);
-                        else tma_load_2d(smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES), &tmap, kc * 64, tap * cout_pad + tl.n0, full);
+                        const uint32_t dst = smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES);
+                        if (CG == 2) {       // this CTA's half of the rows; completion is reported to the leader's barrier
+                            const uint32_t full = leader_bar(&bars->b_full[stage]);
+                            const int row0 = tl.n0 + (int)rank * (BN / 2);
+                            mbar_arrive_expect_tx_cluster(full, Cfg::B_STAGE_BYTES);
+                            if (second) tma_load_2d_pair(dst, &tmap2, (kc - kchunks) * 64, row0, full);
+                            else tma_load_2d_pair(dst, &tmap, kc * 64, tap * cout_pad + row0, full);
+                        } else {
+                            const uint32_t full = smem_u32(&bars->b_full[stage]);
+                            mbar_arrive_expect_tx(full, Cfg::B_STAGE_BYTES);
+                            if (second) tma_load_2d(dst, &tmap2, (kc - kchunks) * 64, tl.n0, full);
+                            else tma_load_2d(dst, &tmap, kc * 64, tap * cout_pad + tl.n0, full);
+                        }
                         ++issued;
                         if (++stage == Cfg::B_STAGES) { stage = 0; phase ^= 1; }
                     }
@@ -523,7 +627,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
             }
         }
-    } else if (warp == MMA_WARP || (PAIR == 2 && warp == MMA_WARP2)) {
+    } else if ((warp == MMA_WARP && rank == 0) || (PAIR == 2 && warp == MMA_WARP2)) {
         // ------------------------------------------------ MMA issue
         // The whole warp runs the loop and one elected lane issues: in warp-uniform code the
         // compiler keeps descriptors and counters in uniform registers, and the issue sequence of
@@ -535,9 +639,18 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         {
             const int me = warp == MMA_WARP ? 0 : 1;          // the tile slot this warp issues for
             const bool leader = elect_one() != 0u;
-            constexpr uint32_t idesc = make_idesc_bf16(128, BN);
+            constexpr uint32_t idesc = make_idesc_bf16(128 * CG, BN);
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
             const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)) + me * (A_TILE_BYTES >> 4), b_lo0 = desc_lo(smem_u32(smem_b));
+            // one MMA of the pair (M = 256 over both CTAs) or of this CTA; a commit to both CTAs or to this one
+            auto mma = [&](uint32_t d, uint32_t alo, uint32_t blo, uint32_t accum) {
+                if (CG == 2) umma2_bf16_split(d, alo, a_hi, blo, b_hi, idesc, accum);
+                else umma_bf16_split(d, alo, a_hi, blo, b_hi, idesc, accum);
+            };
+            auto commit = [&](uint64_t* b) {
+                if (CG == 2) umma2_commit_both(smem_u32(b));
+                else umma_commit(smem_u32(b));
+            };
             Tracer tr; tr.init((me == 0 && lane == 0) ? a.trace : nullptr, 1);
             tr.mark_at(40, t_entry);
             tr.mark(41);
@@ -545,7 +658,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             bool ok = true;
             int n_item = 0;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
-                const int cnt = sched.count(t);
+                const int n = sched.count(t);
+                const int cnt = sched.mine(n);
                 const bool active = me < cnt;
                 const int buf = n_item % NBUF;
                 tr.mark(20);
@@ -577,14 +691,14 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
                         if (leader) {
                             if (active) {
-                                umma_bf16_split(td, a_lo, a_hi, b_lo, b_hi, idesc, acc);
-                                umma_bf16_split(td, a_lo + 2, a_hi, b_lo + 2, b_hi, idesc, 1u);
-                                umma_bf16_split(td, a_lo + 4, a_hi, b_lo + 4, b_hi, idesc, 1u);
-                                umma_bf16_split(td, a_lo + 6, a_hi, b_lo + 6, b_hi, idesc, 1u);
+                                mma(td, a_lo, b_lo, acc);
+                                mma(td, a_lo + 2, b_lo + 2, 1u);
+                                mma(td, a_lo + 4, b_lo + 4, 1u);
+                                mma(td, a_lo + 6, b_lo + 6, 1u);
                             }
                             // weight stages are handed back B_GROUP at a time (fewer commits)
                             if (bs % Cfg::B_GROUP == Cfg::B_GROUP - 1) {
-                                if (active) umma_commit(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
+                                if (active) commit(&bars->b_empty[bs / Cfg::B_GROUP]);
                                 else mbar_arrive(smem_u32(&bars->b_empty[bs / Cfg::B_GROUP]));
                             }
                         }
@@ -594,24 +708,25 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         if (++kx == 3) { kx = 0; a_lo += (PW - 2) * 8; } else a_lo += 8;
                     }
                     if (leader) {
-                        if (active) umma_commit(smem_u32(&bars->a_empty[as]));
+                        if (active) commit(&bars->a_empty[as]);
                         else mbar_arrive(smem_u32(&bars->a_empty[as]));
                     }
                     __syncwarp();
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
                 if (ok && leader) {
-                    if (active) umma_commit(smem_u32(&bars->acc_full[buf]));
+                    if (active) commit(&bars->acc_full[buf]);
                     else mbar_arrive(smem_u32(&bars->acc_full[buf]));
                 }
                 __syncwarp();
-                t += cnt;
+                t += n;
             }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();                         // nobody leaves while the pair may still touch its memory
     if (tid == 0 && bars->abort_flag && status) {
         if (atomicCAS(status, 0u, 0xC0DE0001u) == 0u) {
             status[1] = blockIdx.x;
@@ -620,7 +735,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     }
     if (warp == MMA_WARP) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, (uint32_t)Cfg::TMEM_COLS);
+        if (CG == 2) tmem_dealloc2(tmem_base, (uint32_t)Cfg::TMEM_COLS);
+        else tmem_dealloc(tmem_base, (uint32_t)Cfg::TMEM_COLS);
     }
 }
 
@@ -677,21 +793,65 @@ int num_sms() {
     return n;
 }
 
-template <int BN, bool IB, int OM>
+// clusters of two CTAs of this kernel that the device can hold at once (0: the form cannot run)
+template <typename K>
+int max_pairs(K kern, int smem) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, (const void*)kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
+template <int BN, bool IB, int OM, int CG>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM>;
+    auto kern = conv_tc_kernel<BN, IB, OM, CG>;
+    constexpr int SMEM = TileCfg<BN, CG>::SMEM_TOTAL;
     static bool configured = false;
+    static int pairs = 0;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<BN>::SMEM_TOTAL);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
+        if (CG == 2) {
+            pairs = max_pairs(kern, SMEM);
+            if (pairs < 1) return cudaErrorInvalidConfiguration;
+        }
         configured = true;
     }
     const int tiles = ((a.W + TILE_W - 1) / TILE_W) * ((a.H + TILE_H - 1) / TILE_H);
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
-    int grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
-    if (getenv("VD_CONV_GRID")) grid = std::min(grid, atoi(getenv("VD_CONV_GRID")));   // timing studies
-    return launch_pdl(kern, dim3(grid), dim3(NUM_THREADS), TileCfg<BN>::SMEM_TOTAL, s, a, *(const CUtensorMap*)plan.tmap,
-                      *(const CUtensorMap*)plan.tmap2, *(const CUtensorMap*)plan.tmap_y, status);
+    int grid;
+    if (CG == 2) grid = 2 * (int)std::min<long long>((total + 1) / 2, std::min(pairs, kConvMaxCtas / 2));
+    else grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
+    if (getenv("VD_CONV_GRID")) grid = std::max(CG, std::min(grid, atoi(getenv("VD_CONV_GRID")) / CG * CG));   // timing studies
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (pdl_enabled()) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    if (CG == 2) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kern, a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
+                              *(const CUtensorMap*)plan.tmap_y, status);
 }
 
 }  // namespace
@@ -727,9 +887,14 @@ cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int 
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     const int taps = a.ksize * a.ksize;
     const int bn = pick_bn(a.Cout);
-    if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, taps * padded_cout(a.Cout), bn)) return cudaErrorInvalidValue;
+    // 256-channel blocks run as two-CTA pairs (each CTA loads half of the rows of a weight tile)
+    static const char* pairs_env = getenv("VD_CONV_PAIRS");                 // timing studies: none | up | all
+    const int pairs_mode = !pairs_env ? 1 : (pairs_env[0] == 'n' ? 0 : (pairs_env[0] == 'a' ? 2 : 1));
+    const int cg = (bn == 256 && (pairs_mode == 2 || (pairs_mode == 1 && a.upsample))) ? 2 : 1;
+    plan->cg = cg;
+    if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, taps * padded_cout(a.Cout), bn / cg)) return cudaErrorInvalidValue;
     if (a.x2) {
-        if (!encode_weights((CUtensorMap*)plan->tmap2, a.w2, a.Cin2, a.Cout, bn)) return cudaErrorInvalidValue;
+        if (!encode_weights((CUtensorMap*)plan->tmap2, a.w2, a.Cin2, a.Cout, bn / cg)) return cudaErrorInvalidValue;
     } else {
         memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
     }
@@ -767,18 +932,24 @@ cudaError_t launch_conv_tc(const ConvArgs& a_in, const ConvTcPlan& plan, unsigne
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.bn == 16) {
-        return ib ? launch_one<16, true, 2>(a, plan, status, s) : launch_one<16, false, 2>(a, plan, status, s);
+        return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
+    }
+    if (plan.bn == 256 && plan.cg == 2) {
+        if (ib && ob) return launch_one<256, true, 1, 2>(a, plan, status, s);
+        if (ib && !ob) return launch_one<256, true, 0, 2>(a, plan, status, s);
+        if (!ib && ob) return launch_one<256, false, 1, 2>(a, plan, status, s);
+        return launch_one<256, false, 0, 2>(a, plan, status, s);
     }
     if (plan.bn == 256) {
-        if (ib && ob) return launch_one<256, true, 1>(a, plan, status, s);
-        if (ib && !ob) return launch_one<256, true, 0>(a, plan, status, s);
-        if (!ib && ob) return launch_one<256, false, 1>(a, plan, status, s);
-        return launch_one<256, false, 0>(a, plan, status, s);
+        if (ib && ob) return launch_one<256, true, 1, 1>(a, plan, status, s);
+        if (ib && !ob) return launch_one<256, true, 0, 1>(a, plan, status, s);
+        if (!ib && ob) return launch_one<256, false, 1, 1>(a, plan, status, s);
+        return launch_one<256, false, 0, 1>(a, plan, status, s);
     }
-    if (ib && ob) return launch_one<128, true, 1>(a, plan, status, s);
-    if (ib && !ob) return launch_one<128, true, 0>(a, plan, status, s);
-    if (!ib && ob) return launch_one<128, false, 1>(a, plan, status, s);
-    return launch_one<128, false, 0>(a, plan, status, s);
+    if (ib && ob) return launch_one<128, true, 1, 1>(a, plan, status, s);
+    if (ib && !ob) return launch_one<128, true, 0, 1>(a, plan, status, s);
+    if (!ib && ob) return launch_one<128, false, 1, 1>(a, plan, status, s);
+    return launch_one<128, false, 0, 1>(a, plan, status, s);
 }
 
 }  // namespace vd

@@ -97,6 +97,7 @@ struct alignas(64) ConvTcPlan {
     void* y;                    // the output address tmap_y was built for
     int batch;                  // frames covered by tmap_y
     int bn;
+    int cg;                     // CTAs per MMA: 2 = two-CTA pairs (weight maps built with half-height boxes)
     int valid;
 };
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
