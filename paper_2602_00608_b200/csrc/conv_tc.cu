@@ -64,7 +64,7 @@ template <int BN, int CG = 1> struct TileCfg {
     static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
     static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 6 : 8));
-    static constexpr int B_GROUP = 2;                                // weight stages handed back per tcgen05.commit
+    static constexpr int B_GROUP = BN == 256 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = CG == 2 ? 3 : 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
