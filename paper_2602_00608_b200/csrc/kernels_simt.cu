@@ -428,8 +428,71 @@ cudaError_t launch_gn_stats(const GnArgs& a, cudaStream_t s) {
     return cudaGetLastError();
 }
 
+// The first convolution (latent channels -> hundreds of channels): K = 9 * Cin <= 72 is too thin for the
+// tensor core and for the tiled FFMA kernel's staging.  A block computes 32 consecutive pixels x 128
+// output channels: the pixels' 3x3 neighbourhoods sit in shared memory, a thread holds 4 pixels x 4
+// channels and reads the weights ([tap][Cin][Cout] fp32) as coalesced float4 straight from L1/L2.
+constexpr int kThinPix = 32, kThinCout = 128, kThinMaxK = 72;
+template <int CIN>
+__global__ void __launch_bounds__(256) conv_thin_kernel(ConvArgs a) {
+    __shared__ float in_s[kThinPix][kThinMaxK + 1];
+    griddep_launch();
+    griddep_wait();
+    constexpr int K = 9 * CIN;
+    const long long npix = (long long)a.B * a.H * a.W;
+    const long long p0 = (long long)blockIdx.x * kThinPix;
+    const int co0 = blockIdx.y * kThinCout;
+    const float* x = (const float*)a.x;
+    for (int i = threadIdx.x; i < kThinPix * K; i += 256) {
+        const int p = i / K, k = i - p * K;
+        const int tap = k / CIN, c = k - tap * CIN;
+        const long long g = p0 + p;
+        float v = 0.f;
+        if (g < npix) {
+            const int b = (int)(g / ((long long)a.H * a.W));
+            const int r = (int)(g - (long long)b * a.H * a.W);
+            const int oy = r / a.W + tap / 3 - 1, ox = r % a.W + tap % 3 - 1;
+            if (oy >= 0 && oy < a.H && ox >= 0 && ox < a.W) v = x[(((size_t)b * a.H + oy) * a.W + ox) * CIN + c];
+        }
+        in_s[p][k] = a.bf16_operands ? round_bf16(v) : v;
+    }
+    __syncthreads();
+    const int pg = threadIdx.x >> 5, cg = threadIdx.x & 31;          // 4 pixels, 4 channels per thread
+    const float* w = (const float*)a.w + co0 + cg * 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[i][q] = 0.f;
+#pragma unroll 12
+    for (int k = 0; k < K; ++k) {
+        const float4 wv = __ldg((const float4*)(w + (size_t)k * a.Cout));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float xv = in_s[pg * 4 + i][k];
+            acc[i][0] = fmaf(xv, wv.x, acc[i][0]); acc[i][1] = fmaf(xv, wv.y, acc[i][1]);
+            acc[i][2] = fmaf(xv, wv.z, acc[i][2]); acc[i][3] = fmaf(xv, wv.w, acc[i][3]);
+        }
+    }
+    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.bias) bv = __ldg((const float4*)(a.bias + co0 + cg * 4));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const long long g = p0 + pg * 4 + i;
+        if (g < npix)
+            *(float4*)((float*)a.y + (size_t)g * a.Cout + co0 + cg * 4) =
+                make_float4(acc[i][0] + bv.x, acc[i][1] + bv.y, acc[i][2] + bv.z, acc[i][3] + bv.w);
+    }
+}
+
 cudaError_t launch_conv_simt(const ConvArgs& a, cudaStream_t s) {
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
+    if (!ib && !ob && a.ksize == 3 && (a.Cin == 4 || a.Cin == 8) && a.Cout % kThinCout == 0 && !a.scale && !a.residual &&
+        !a.upsample && !a.out_nchw && !a.x2) {
+        const long long npix = (long long)a.B * a.H * a.W;
+        dim3 grid((unsigned)((npix + kThinPix - 1) / kThinPix), a.Cout / kThinCout);
+        return a.Cin == 4 ? launch_pdl(conv_thin_kernel<4>, grid, dim3(256), 0, s, a) : launch_pdl(conv_thin_kernel<8>, grid, dim3(256), 0, s, a);
+    }
     if (ib && ob) return conv_simt_dispatch<__nv_bfloat16, __nv_bfloat16>(a, s);
     if (ib && !ob) return conv_simt_dispatch<__nv_bfloat16, float>(a, s);
     if (!ib && ob) return conv_simt_dispatch<float, __nv_bfloat16>(a, s);
