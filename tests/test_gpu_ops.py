@@ -187,6 +187,10 @@ TC_CASES = [
     dict(B=1, H=17, W=16, Cin=512, Cout=512, k=3, upsample=False, prologue=True, silu=True, residual=True, in_bf16=True, out_bf16=False),
     dict(B=2, H=37, W=21, Cin=128, Cout=3, k=3, upsample=False, prologue=True, silu=True, residual=False, in_bf16=False, out_bf16=True, out_nchw=True),
     dict(B=3, H=50, W=70, Cin=128, Cout=128, k=3, upsample=False, prologue=True, silu=True, residual=True, in_bf16=True, out_bf16=False),
+    # upsampling layers with 256-channel blocks run as two-CTA pairs: an odd number of tiles per channel block
+    # (the peer CTA of the last pair has no tile), two channel blocks, two frames
+    dict(B=1, H=17, W=9, Cin=64, Cout=256, k=3, upsample=True, prologue=False, silu=False, residual=False, in_bf16=False, out_bf16=False),
+    dict(B=2, H=12, W=11, Cin=128, Cout=512, k=3, upsample=True, prologue=True, silu=True, residual=False, in_bf16=False, out_bf16=True),
 ]
 
 
