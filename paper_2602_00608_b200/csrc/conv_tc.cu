@@ -63,15 +63,17 @@ template <int BN, int CG = 1> struct TileCfg {
     static_assert(CG == 1 || BN == 256, "the two-CTA form exists for 256-channel blocks only");
     static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
-    static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 6 : 8));
-    static constexpr int B_GROUP = BN == 256 ? 1 : 2;                // weight stages handed back per tcgen05.commit
+    static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 3 : 8));
+    static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = CG == 2 ? 3 : 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
     static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
-    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + 512 + 1024;  // + barriers + alignment slack
+    // two-tile items: the producers stage the raw input of the next unit in shared memory (cp.async)
+    static constexpr int SMEM_RAW = PAIR == 2 ? ITEMS * 32 : 0;
+    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + 512 + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
     static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
@@ -177,6 +179,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     uint8_t* smem_a = smem_out + Cfg::SMEM_OUT;
     uint8_t* smem_bias = smem_a + Cfg::SMEM_A;
     Bars* bars = (Bars*)(smem_bias + Cfg::SMEM_BIAS);
+    uint8_t* smem_stage = smem_bias + Cfg::SMEM_BIAS + 512;  // raw input of the next unit (two-tile items only)
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const long long t_entry = Tracer::now();
@@ -264,6 +267,164 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         Tracer tr; tr.init(ptid == 0 ? a.trace : nullptr, 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
+        if constexpr (PAIR == 2) {
+            // Two-tile items (narrow channel blocks) are bound by this role, and a thread's registers hold
+            // one unit of input only.  So the raw input of the NEXT unit travels by cp.async into a
+            // shared-memory staging area while the current unit is transformed: every thread copies exactly
+            // the entries it later reads back (16-byte pieces at [half][entry][thread]), so the staging needs
+            // no synchronisation between threads, and invalid entries are zero-filled by the copy.
+            struct Pos { int t, cnt, kc, slot; Tile tile; };      // tile = tile (t + slot)
+            auto advance = [&](Pos& p) {
+                if (++p.slot < p.cnt) {                          // the item's second tile: the next one of its channel block
+                    p.tile.tx0 += TILE_W;
+                    if (p.tile.tx0 >= sched.tiles_x * TILE_W) { p.tile.tx0 = 0; p.tile.ty0 += TILE_H; }
+                    return;
+                }
+                const bool two = p.slot == 2;
+                p.slot = 0;
+                if (++p.kc < ktotal) {                           // next chunk of the same item: back to its first tile
+                    if (two) {
+                        if (p.tile.tx0 == 0) { p.tile.tx0 = (sched.tiles_x - 1) * TILE_W; p.tile.ty0 -= TILE_H; }
+                        else p.tile.tx0 -= TILE_W;
+                    }
+                    return;
+                }
+                p.kc = 0;
+                p.t += p.cnt;
+                if (p.t < sched.end) { p.cnt = sched.count(p.t); p.tile = sched.get(p.t, BN); }
+            };
+            const uint32_t st_lo = smem_u32(smem_stage) + (uint32_t)ptid * 16u;           // + u * NUM_PRODUCERS * 16
+            const uint32_t st_hi = st_lo + (uint32_t)(ITEMS * 16);
+            // starts the copies of unit p; returns which of this thread's entries exist
+            auto issue = [&](const Pos& p) -> uint32_t {
+                const bool second = p.kc >= kchunks;
+                const int c0 = (second ? p.kc - kchunks : p.kc) * 64;
+                const bool centre_only = second || a.ksize == 1;
+                const Tile& tile = p.tile;
+                uint32_t vm = 7u;
+                const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
+                if (!interior || centre_only) {
+                    vm = 0u;
+#pragma unroll
+                    for (int u = 0; u < BATCH; ++u) {
+                        const int oy = tile.ty0 + (int)(pyx[u] & 0xffu) - 1, ox = tile.tx0 + (int)((pyx[u] >> 8) & 0xffu) - 1;
+                        bool v = oy >= 0 && oy < a.H && ox >= 0 && ox < a.W;
+                        if (centre_only) v = v && (pyx[u] >> 16) != 0u;
+                        vm |= (v ? 1u : 0u) << u;
+                    }
+                }
+                if (!second) {
+                    const char* xb = (const char*)a.x
+                        + ((((size_t)tile.b * a.Hs + (tile.ty0 >> up)) * a.Ws + (tile.tx0 >> up)) * a.Cin + c0 + (IN_BF16 ? j * 8 : j * 4)) * ESZ;
+#pragma unroll
+                    for (int u = 0; u < BATCH; ++u) {
+                        const bool v = (vm >> u) & 1u;
+                        const char* src = v ? xb + goff[u] : (const char*)a.x;
+                        cp_async16(st_lo + (uint32_t)(u * NUM_PRODUCERS * 16), src, v ? 16u : 0u);
+                        if (!IN_BF16) cp_async16(st_hi + (uint32_t)(u * NUM_PRODUCERS * 16), src + (v ? 128 : 0), v ? 16u : 0u);
+                    }
+                } else {             // fused shortcut: fp32 input at the output resolution, centre pixels only
+                    const char* xb = (const char*)a.x2 + ((((size_t)tile.b * a.H + tile.ty0) * a.W + tile.tx0) * a.Cin2 + c0 + j * 4) * 4;
+#pragma unroll
+                    for (int u = 0; u < BATCH; ++u) {
+                        const bool v = (vm >> u) & 1u;
+                        const char* src = v ? xb + (((int)(pyx[u] & 0xffu) - 1) * a.W + ((int)((pyx[u] >> 8) & 0xffu) - 1)) * a.Cin2 * 4 : (const char*)a.x2;
+                        cp_async16(st_lo + (uint32_t)(u * NUM_PRODUCERS * 16), src, v ? 16u : 0u);
+                        cp_async16(st_hi + (uint32_t)(u * NUM_PRODUCERS * 16), src + (v ? 128 : 0), v ? 16u : 0u);
+                    }
+                }
+                cp_async_commit();
+                return vm;
+            };
+            float sc[8], sh[8];
+            auto load_affine = [&](const Pos& p) {               // GroupNorm scale/shift of the unit's channels
+                if (!prologue || p.kc >= kchunks) return;
+                // channels of v[0..3] and v[4..7] (see load_raw); the tiles of an item lie in one frame
+                const int ca = p.kc * 64 + (IN_BF16 ? j * 8 : j * 4), cb = IN_BF16 ? ca + 4 : ca + 32;
+                const float* ps = a.scale + (size_t)p.tile.b * a.Cin;
+                const float* pt = a.shift + (size_t)p.tile.b * a.Cin;
+                const float4 s0 = __ldg((const float4*)(ps + ca)), s1 = __ldg((const float4*)(ps + cb));
+                const float4 t0 = __ldg((const float4*)(pt + ca)), t1 = __ldg((const float4*)(pt + cb));
+                sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
+                sh[0] = t0.x; sh[1] = t0.y; sh[2] = t0.z; sh[3] = t0.w; sh[4] = t1.x; sh[5] = t1.y; sh[6] = t1.z; sh[7] = t1.w;
+                if (silu) {          // SiLU is evaluated as h + h*tanh(h) with h = v/2: the 1/2 folds into the affine map
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { sc[e] *= 0.5f; sh[e] *= 0.5f; }
+                }
+            };
+            Pos nx;
+            nx.t = sched.begin; nx.kc = 0; nx.slot = 0; nx.cnt = 1;
+            bool have = nx.t < sched.end;
+            uint32_t vm_next = 0u;
+            if (have) {
+                nx.cnt = sched.count(nx.t);
+                nx.tile = sched.get(nx.t, BN);
+                vm_next = issue(nx);
+                load_affine(nx);
+            }
+            while (have && ok) {
+                const int cur_kc = nx.kc, cur_slot = nx.slot, cur_cnt = nx.cnt, cur_t = nx.t;
+                const uint32_t cur_vm = vm_next;
+                const bool second = cur_kc >= kchunks;
+                const bool pro = prologue && !second;
+                const bool in_bf16 = IN_BF16 && !second;
+                advance(nx);
+                const bool have_next = nx.t < sched.end;
+                tr.mark(1);
+                cp_async_wait_all();                             // this thread's pieces of the current unit have landed
+                Raw8 raw[BATCH];
+#pragma unroll
+                for (int u = 0; u < BATCH; ++u) {
+                    raw[u].lo = lds_u4(st_lo + (uint32_t)(u * NUM_PRODUCERS * 16));
+                    if (!in_bf16) raw[u].hi = lds_u4(st_hi + (uint32_t)(u * NUM_PRODUCERS * 16));
+                }
+                if (have_next) vm_next = issue(nx);              // the staging slots are free again: the next unit is on its way
+                if (cur_slot == 0) {
+                    ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
+                    if (!ok) break;
+                }
+                tr.mark(2);
+                uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur_slot * A_TILE_BYTES;
+#pragma unroll
+                for (int u = 0; u < BATCH; ++u) {
+                    uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
+                    if (cur_vm & (1u << u)) {
+                        float v[8];
+                        unpack_raw(in_bf16, raw[u], v);
+                        if (pro) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], sc[e], sh[e]);
+                            if (silu) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], tanh_fast(v[e]), v[e]);
+                            }
+                        }
+                        o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]);
+                    }
+                    if (in_bf16) {
+                        *(uint4*)(dst_tile + soff[u]) = make_uint4(o0, o1, o2, o3);
+                    } else {
+                        uint32_t so = soff[u];
+                        if (IN_BF16) {                           // fp32 second input of a kernel whose first input is bf16
+                            const uint32_t pix = so >> 7;
+                            so = pix * 128 + (((j >> 1) ^ (pix & 7)) << 4) + (j & 1) * 8;
+                        }
+                        *(uint2*)(dst_tile + so) = make_uint2(o0, o1);
+                        *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
+                    }
+                }
+                if (cur_slot == cur_cnt - 1) {
+                    fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[stage]));
+                    if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (have_next && (nx.kc != cur_kc || nx.t != cur_t)) load_affine(nx);
+                tr.mark(3);
+                have = have_next;
+            }
+            cp_async_wait_all();
+        } else
         for (int t = sched.begin; t < sched.end && ok;) {
             const int n = sched.count(t);
             const int cnt = sched.mine(n);                   // 0: the peer of a two-CTA pair in an odd tail item
