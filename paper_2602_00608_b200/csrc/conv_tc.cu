@@ -233,7 +233,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     griddep_launch();
 
     if (is_producer_warp(warp)) {
-        griddep_wait();
         // ------------------------------------------------ operand prologue (producers)
         // The work is a sequence of units (item, chunk, tile slot); a thread owns three (pixel,
         // 8-channel group) entries of every unit, all loaded before any is consumed.  The role is
@@ -267,6 +266,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         Tracer tr; tr.init(ptid == 0 ? a.trace : nullptr, 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
+        griddep_wait();              // everything above is arithmetic on the thread's own indices
         if constexpr (PAIR == 2) {
             // Two-tile items (narrow channel blocks) are bound by this role, and a thread's registers hold
             // one unit of input only.  So the raw input of the NEXT unit travels by cp.async into a
@@ -1051,7 +1051,17 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     // 256-channel blocks run as two-CTA pairs (each CTA loads half of the rows of a weight tile)
     static const char* pairs_env = getenv("VD_CONV_PAIRS");                 // timing studies: none | up | all
     const int pairs_mode = !pairs_env ? 1 : (pairs_env[0] == 'n' ? 0 : (pairs_env[0] == 'a' ? 2 : 1));
-    const int cg = (bn == 256 && (pairs_mode == 2 || (pairs_mode == 1 && a.upsample))) ? 2 : 1;
+    int cg = (bn == 256 && (pairs_mode == 2 || (pairs_mode == 1 && a.upsample))) ? 2 : 1;
+    if (cg == 2) {       // the device must be able to co-schedule pairs of these CTAs; else the one-CTA form
+        static int probe = -1;
+        if (probe < 0) {
+            auto k = conv_tc_kernel<256, false, 1, 2>;
+            probe = (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<256, 2>::SMEM_TOTAL) == cudaSuccess)
+                        ? max_pairs(k, TileCfg<256, 2>::SMEM_TOTAL) : 0;
+            cudaGetLastError();
+        }
+        if (probe < 1) cg = 1;
+    }
     plan->cg = cg;
     if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, taps * padded_cout(a.Cout), bn / cg)) return cudaErrorInvalidValue;
     if (a.x2) {
