@@ -65,14 +65,15 @@ template <int BN, int CG = 1> struct TileCfg {
     static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
     static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 3 : 8));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
-    static constexpr int A_STAGES = CG == 2 ? 3 : 2;
+    static constexpr int A_STAGES = 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
     static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
-    // two-tile items: the producers stage the raw input of the next unit in shared memory (cp.async)
-    static constexpr int SMEM_RAW = PAIR == 2 ? ITEMS * 32 : 0;
+    // two-tile items and two-CTA pairs: the producers stage the raw input of the next unit in shared memory (cp.async)
+    static constexpr bool STAGED = PAIR == 2 || CG == 2;
+    static constexpr int SMEM_RAW = STAGED ? ITEMS * 32 : 0;
     static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + 512 + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
@@ -267,13 +268,18 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         griddep_wait();              // everything above is arithmetic on the thread's own indices
-        if constexpr (PAIR == 2) {
-            // Two-tile items (narrow channel blocks) are bound by this role, and a thread's registers hold
+        if constexpr (Cfg::STAGED) {
+            // Two-tile items (narrow channel blocks) and two-CTA pairs are bound by this role, and a thread's registers hold
             // one unit of input only.  So the raw input of the NEXT unit travels by cp.async into a
             // shared-memory staging area while the current unit is transformed: every thread copies exactly
             // the entries it later reads back (16-byte pieces at [half][entry][thread]), so the staging needs
             // no synchronisation between threads, and invalid entries are zero-filled by the copy.
-            struct Pos { int t, cnt, kc, slot; Tile tile; };      // tile = tile (t + slot)
+            struct Pos { int t, n, cnt, kc, slot; Tile tile; };   // n tiles in the item, cnt of them this CTA's; tile = its slot-th
+            auto first_of_item = [&](Pos& p) {
+                p.n = sched.count(p.t);
+                p.cnt = sched.mine(p.n);                         // 0: the peer of a two-CTA pair in an odd tail item
+                p.tile = sched.get(p.cnt > 0 ? sched.index(p.t, 0) : p.t, BN);
+            };
             auto advance = [&](Pos& p) {
                 if (++p.slot < p.cnt) {                          // the item's second tile: the next one of its channel block
                     p.tile.tx0 += TILE_W;
@@ -290,8 +296,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     return;
                 }
                 p.kc = 0;
-                p.t += p.cnt;
-                if (p.t < sched.end) { p.cnt = sched.count(p.t); p.tile = sched.get(p.t, BN); }
+                p.t += p.n;
+                if (p.t < sched.end) first_of_item(p);
             };
             const uint32_t st_lo = smem_u32(smem_stage) + (uint32_t)ptid * 16u;           // + u * NUM_PRODUCERS * 16
             const uint32_t st_hi = st_lo + (uint32_t)(ITEMS * 16);
@@ -301,6 +307,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const int c0 = (second ? p.kc - kchunks : p.kc) * 64;
                 const bool centre_only = second || a.ksize == 1;
                 const Tile& tile = p.tile;
+                if (p.cnt == 0) { cp_async_commit(); return 0u; }  // no tile of this CTA in the item: nothing to copy
                 uint32_t vm = 7u;
                 const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
                 if (!interior || centre_only) {
@@ -353,17 +360,17 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
             };
             Pos nx;
-            nx.t = sched.begin; nx.kc = 0; nx.slot = 0; nx.cnt = 1;
+            nx.t = sched.begin; nx.kc = 0; nx.slot = 0; nx.cnt = 1; nx.n = 1;
             bool have = nx.t < sched.end;
             uint32_t vm_next = 0u;
             if (have) {
-                nx.cnt = sched.count(nx.t);
-                nx.tile = sched.get(nx.t, BN);
+                first_of_item(nx);
                 vm_next = issue(nx);
                 load_affine(nx);
             }
             while (have && ok) {
                 const int cur_kc = nx.kc, cur_slot = nx.slot, cur_cnt = nx.cnt, cur_t = nx.t;
+                const bool cur_have = cur_cnt > 0;               // without a tile the CTA still follows the barriers
                 const uint32_t cur_vm = vm_next;
                 const bool second = cur_kc >= kchunks;
                 const bool pro = prologue && !second;
@@ -387,6 +394,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur_slot * A_TILE_BYTES;
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
+                    if (!cur_have) break;
                     uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
                     if (cur_vm & (1u << u)) {
                         float v[8];
@@ -413,10 +421,10 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
                     }
                 }
-                if (cur_slot == cur_cnt - 1) {
+                if (cur_slot >= cur_cnt - 1) {
                     fence_proxy_async_smem();                    // generic-proxy stores -> visible to the tensor core
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[stage]));
+                    if (lane == 0) arrive_leader(&bars->a_full[stage]);
                     if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (have_next && (nx.kc != cur_kc || nx.t != cur_t)) load_affine(nx);
