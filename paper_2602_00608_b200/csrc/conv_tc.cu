@@ -596,10 +596,12 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             uint8_t* wout = smem_out + ew * (2 * WARP_SLICE_BYTES);         // this warp's two slice buffers
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
             int bias_n0 = -1;
+            constexpr int TAIL_BUFS = Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) >= 2 ? Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) : 2;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int n = sched.count(t);
                 const int cnt = sched.mine(n);
                 const int buf = n_item % NBUF;
+                const bool last_item = t + n >= sched.end && Cfg::SMEM_B >= 8 * WARP_SLICE_BYTES;
                 tr.mark(10);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
                 if (!ok) break;
@@ -631,9 +633,15 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         uint32_t (&rn)[32] = (p & 1) ? ra : rb;          // next pass, in flight while this one is processed
                         if (p + 1 < NP) tmem_ld32(tacc + (uint32_t)((p + 1) * 32), rn);
                         const int sl = p / PPS, h = p % PPS;              // slice, half of the slice
-                        uint8_t* obuf = wout + ((n_slice + sl) & 1) * WARP_SLICE_BYTES;
+                        // The CTA's last item has the weight stages to itself (every MMA has completed): its slices go
+                        // through a longer ring of buffers there, so the stores of the tail are not paced by buffer reuse.
+                        uint8_t* obuf = last_item ? smem_b + (ew * TAIL_BUFS + (int)((n_slice + sl) % TAIL_BUFS)) * WARP_SLICE_BYTES
+                                                  : wout + ((n_slice + sl) & 1) * WARP_SLICE_BYTES;
                         if (h == 0) {
-                            if (lane == 0) bulk_wait_group_read<1>();     // the store that last read this buffer is done
+                            if (lane == 0) {                              // the store that last read this buffer is done
+                                if (last_item) bulk_wait_group_read<TAIL_BUFS - 1>();
+                                else bulk_wait_group_read<1>();
+                            }
                             __syncwarp();
                         }
                         uint8_t* orow = obuf + lane * 128;
