@@ -69,6 +69,10 @@ SIMT_CASES = [
     dict(B=2, H=10, W=17, Cin=24, Cout=12, k=1, upsample=False, prologue=True, silu=False, residual=True),
     dict(B=1, H=33, W=21, Cin=32, Cout=3, k=3, upsample=False, prologue=True, silu=True, residual=False, out_nchw=True),
     dict(B=1, H=5, W=6, Cin=4, Cout=64, k=3, upsample=False, prologue=False, silu=False, residual=False),
+    # thin first-convolution kernel (K = 9 * Cin <= 72, Cout a multiple of 128): pixel count not a multiple of 32,
+    # two frames, both supported input widths
+    dict(B=2, H=7, W=9, Cin=4, Cout=128, k=3, upsample=False, prologue=False, silu=False, residual=False),
+    dict(B=1, H=13, W=5, Cin=8, Cout=256, k=3, upsample=False, prologue=False, silu=False, residual=False),
 ]
 
 
