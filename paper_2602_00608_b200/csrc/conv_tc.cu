@@ -1021,7 +1021,8 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     int grid;
     if (CG == 2) grid = 2 * (int)std::min<long long>((total + 1) / 2, std::min(pairs, kConvMaxCtas / 2));
     else grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
-    if (getenv("VD_CONV_GRID")) grid = std::max(CG, std::min(grid, atoi(getenv("VD_CONV_GRID")) / CG * CG));   // timing studies
+    static const int grid_cap = getenv("VD_CONV_GRID") ? atoi(getenv("VD_CONV_GRID")) : 0;                      // timing studies
+    if (grid_cap > 0) grid = std::max(CG, std::min(grid, grid_cap / CG * CG));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(NUM_THREADS);
