@@ -63,7 +63,7 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // tensor cycles and SM).  The MMA warp is active in the leader CTA (cluster rank 0) only.  Barriers
 // that gate the MMAs live in the leader: the peer's producers and weight loads signal the leader's
 // "full" barriers across the cluster, its epilogue the leader's "accumulator free" barrier, and the
-// leader's tcgen05.commit multicasts to the "empty" / "accumulator ready" barriers of both CTAs.
+// leader's tcgen05.commit arrives on the "empty" / "accumulator ready" barriers of both CTAs.
 template <int BN, int CG = 1> struct TileCfg {
     static_assert(CG == 1 || BN == 256, "the two-CTA form exists for 256-channel blocks only");
     static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
@@ -156,11 +156,11 @@ __device__ __forceinline__ void umma2_bf16_split(uint32_t d_tmem, uint32_t a_lo,
         "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n}\n"
         ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
-// arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs
+// arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair:
+// one commit to the leader's own barrier, one to the peer's through its cluster address
 __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
-    const uint16_t mask = 3;
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(mask) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_cta(bar, 1)) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc2(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -211,7 +211,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     sched.rank = (int)rank;
 
     if (tid == 0) {
-        // CG = 2: the leader's "full" barriers collect the arrivals of both CTAs; commits are multicast
+        // CG = 2: the leader's "full" barriers collect the arrivals of both CTAs; commits go to both CTAs
         for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), CG * NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), NMMA); }
         for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), CG); mbar_init(smem_u32(&bars->b_empty[i]), NMMA); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), NMMA); mbar_init(smem_u32(&bars->acc_empty[i]), 4 * CG); }
