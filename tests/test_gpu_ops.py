@@ -128,6 +128,35 @@ def test_gn_stats_survive_a_large_common_offset(env):
     np.testing.assert_allclose(sc, wsc, rtol=2e-3)
 
 
+def test_gn_stats_constant_groups_and_reproducibility(env):
+    """Degenerate input (every group constant: variance exactly zero, so rstd = 1/sqrt(eps)), and the
+    properties the one-launch kernel promises: the same bits on every call, and a sample's result does
+    not depend on the batch it is in."""
+    torch, ref, vd, synth = env
+    r = _rng(23)
+    B, H, W, C, G = 3, 37, 29, 64, 8
+    eps = 0.25
+    gamma = r.uniform(0.9, 1.1, C).astype(np.float32)
+    beta = r.uniform(-0.1, 0.1, C).astype(np.float32)
+    const = np.repeat(r.uniform(-5, 5, (B, G)).astype(np.float32), C // G, axis=1)          # [B, C], constant per group
+    x = np.broadcast_to(const[:, :, None, None], (B, C, H, W)).copy()
+    dev = lambda a_: torch.from_numpy(a_).cuda()
+    sc, sh = vd.op_gn_stats(util.nchw_to_dev_nhwc(x, torch.float32), dev(gamma), dev(beta), G, eps)
+    torch.cuda.synchronize()
+    want_sc = np.broadcast_to(gamma / np.float32(math.sqrt(eps)), (B, C))
+    np.testing.assert_allclose(sc.cpu().numpy(), want_sc, rtol=1e-6)
+    np.testing.assert_allclose(sh.cpu().numpy(), beta - const * want_sc, rtol=1e-5, atol=1e-6)
+
+    y = (r.standard_normal((B, C, H, W)) * 2.0 + 0.7).astype(np.float32)
+    yd = util.nchw_to_dev_nhwc(y, torch.float32)
+    a1 = vd.op_gn_stats(yd, dev(gamma), dev(beta), G, 1e-6)
+    a2 = vd.op_gn_stats(yd, dev(gamma), dev(beta), G, 1e-6)
+    one = vd.op_gn_stats(yd[1:2].contiguous(), dev(gamma), dev(beta), G, 1e-6)
+    torch.cuda.synchronize()
+    assert torch.equal(a1[0], a2[0]) and torch.equal(a1[1], a2[1])
+    assert torch.equal(a1[0][1:2], one[0]) and torch.equal(a1[1][1:2], one[1])
+
+
 def _attn_case(env, seed, B, T, C, bf16, impl):
     torch, ref, vd, synth = env
     r = _rng(seed)
