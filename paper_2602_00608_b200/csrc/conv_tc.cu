@@ -7,25 +7,29 @@
 // Persistent kernel, one CTA per SM, roles decoupled through mbarrier rings:
 //   * tile = 16x8 output pixels x BN output channels:  D[128 x BN] = sum over taps and 64-channel
 //     chunks of A_tap[128 x 64] * W_tap[64 x BN].  Every CTA owns a contiguous, balanced range of
-//     tiles and walks it in work items of two tiles that share every weight stage.
-//   * 15 producer warps read the raw 18x10-pixel halo tile of a 64-channel chunk from global
-//     memory once, apply
-//     scale/shift (+SiLU), round to bf16 and store it in shared memory in the canonical
-//     un-swizzled K-major layout, as eight planes [8 channels][pixel][16 B].  Every tap is a *view*
-//     of that one tile (descriptor start (ky*10+kx) pixels in; eight-row groups are one tile row
-//     = 10 pixels apart), so the transform runs once per element, not once per tap.
+//     tiles; where BN <= 128 it walks it in work items of two tiles that share every weight stage.
+//   * 15 producer warps (on the SM sub-partitions the MMA warp is not on) read the raw 18x10-pixel
+//     halo tile of a 64-channel chunk once, apply scale/shift (+SiLU), round to bf16 and store it
+//     in shared memory as 180 rows of 128 bytes in the 128-byte-swizzled K-major layout.  Every
+//     tap is a *view* of that one tile (descriptor start (ky*10+kx) rows in; eight-row groups are
+//     one tile row = 10 pixels apart), so the transform runs once per element, not once per tap.
 //     Out-of-image halo pixels are exact zeros (padding applies to the transformed tensor).
+//     For two-tile items and two-CTA pairs the raw input of the next unit is staged in shared
+//     memory by cp.async while the current unit is transformed.
 //     An optional second input (the block's raw input for a width-changing ResNet block) is
 //     appended as extra K with a single centre tap: the 1x1 shortcut without its own round trip.
 //   * 1 warp streams the weights (bf16 [tap][Cout][Cin]) by TMA into 128B-swizzled stages.
-//   * 1 thread issues tcgen05.mma (M=128, N=BN, K=16) into TMEM accumulators (double-buffered
-//     where 4 x BN columns fit).
+//   * 1 warp, running warp-uniform code with one elected lane, issues tcgen05.mma (M=128, N=BN,
+//     K=16) into TMEM accumulators, double-buffered so an item's epilogue overlaps the next item.
 //   * 4 epilogue warps drain the accumulators: tcgen05.ld, + bias, and the tile leaves through
 //     shared memory as 128-byte-wide slices written by bulk tensor stores, which coalesce the
 //     traffic and clip the ragged image edge.  Where the layer has a residual, the output buffer
 //     IS the residual stream and the store is a bulk tensor reduce-add (the fp32 add x + conv(h)
 //     is done once, by the memory system), so the residual never passes through the SM.
 //     The 3-channel frame head writes its NCHW planes directly.
+//   * 1 warp asks L2 ahead of time for the input lines of coming chunks.
+//   * Upsampling layers with 256-channel blocks run as pairs of CTAs (tcgen05.mma.cta_group::2,
+//     see TileCfg).
 // Every wait is bounded: on expiry the CTA records a code in the status word and unwinds.
 #include <cuda.h>
 #include <stdlib.h>
