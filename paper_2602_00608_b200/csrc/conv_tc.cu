@@ -19,8 +19,10 @@
 //     An optional second input (the block's raw input for a width-changing ResNet block) is
 //     appended as extra K with a single centre tap: the 1x1 shortcut without its own round trip.
 //   * 1 warp streams the weights (bf16 [tap][Cout][Cin]) by TMA into 128B-swizzled stages.
-//   * 1 warp, running warp-uniform code with one elected lane, issues tcgen05.mma (M=128, N=BN,
-//     K=16) into TMEM accumulators, double-buffered so an item's epilogue overlaps the next item.
+//   * 1 warp issues tcgen05.mma (M=128, N=BN, K=16) into TMEM accumulators, double-buffered so an
+//     item's epilogue overlaps the next item.  The whole warp runs the loop and the tensor
+//     instructions are predicated on one elected lane (no branch), so the issue sequence is
+//     warp-uniform code with its descriptor arithmetic in uniform registers.
 //   * 4 epilogue warps drain the accumulators: tcgen05.ld, + bias, and the tile leaves through
 //     shared memory as 128-byte-wide slices written by bulk tensor stores, which coalesce the
 //     traffic and clip the ragged image edge.  Where the layer has a residual, the output buffer
@@ -36,6 +38,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "conv_tile.cuh"
 #include "tc_common.cuh"
@@ -72,18 +75,21 @@ template <int BN, int CG = 1> struct TileCfg {
     static_assert(CG == 1 || BN == 256, "the two-CTA form exists for 256-channel blocks only");
     static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
-    static constexpr int B_STAGES = CG == 2 ? 6 : (BN == 256 ? 4 : (BN == 128 ? 3 : 8));
+    static constexpr int OUT_BUFS = 1;                               // output slices per epilogue warp
+    // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
+    static constexpr int B_STAGES = CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
-    static constexpr int SMEM_OUT = BN >= 128 ? 2 * OUT_SLICE_BYTES : 0;   // double-buffered output slices
-    static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES;
+    static constexpr int SMEM_OUT = BN >= 128 ? OUT_BUFS * OUT_SLICE_BYTES : 0;       // output slice(s) per epilogue warp
+    static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES - (A_TILE_BYTES - NPIX * 128);   // the last tile needs no padding
     static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
+    static constexpr int SMEM_BARS = 256;
     // two-tile items and two-CTA pairs: the producers stage the raw input of the next unit in shared memory (cp.async)
     static constexpr bool STAGED = PAIR == 2 || CG == 2;
     static constexpr int SMEM_RAW = STAGED ? ITEMS * 32 : 0;
-    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + 512 + SMEM_RAW + 1024;  // + barriers + alignment slack
+    static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + SMEM_BARS + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
     static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
@@ -160,6 +166,20 @@ __device__ __forceinline__ void umma2_bf16_split(uint32_t d_tmem, uint32_t a_lo,
         "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n}\n"
         ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void umma2_bf16_split_on(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t on) {
+    asm volatile(
+        "{\n.reg .pred p, q;\n.reg .b64 da, db;\nsetp.ne.b32 p, %6, 0;\nsetp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(on) : "memory");
+}
+__device__ __forceinline__ void umma2_commit_both_on(uint32_t bar, uint32_t on) {
+    const uint32_t peer = map_to_cta(bar, 1);
+    asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%1];\n}\n" ::"r"(bar), "r"(peer), "r"(on) : "memory");
+}
 // arrives (once the MMAs issued so far have completed) on the barrier at this offset in both CTAs of the pair:
 // one commit to the leader's own barrier, one to the peer's through its cluster address
 __device__ __forceinline__ void umma2_commit_both(uint32_t bar) {
@@ -190,7 +210,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     uint8_t* smem_a = smem_out + Cfg::SMEM_OUT;
     uint8_t* smem_bias = smem_a + Cfg::SMEM_A;
     Bars* bars = (Bars*)(smem_bias + Cfg::SMEM_BIAS);
-    uint8_t* smem_stage = smem_bias + Cfg::SMEM_BIAS + 512;  // raw input of the next unit (two-tile items only)
+    static_assert(sizeof(Bars) <= Cfg::SMEM_BARS, "barrier block");
+    static_assert(Cfg::SMEM_TOTAL <= 232448, "shared memory of one CTA");
+    uint8_t* smem_stage = smem_bias + Cfg::SMEM_BIAS + Cfg::SMEM_BARS;  // raw input of the next unit (two-tile items only)
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const long long t_entry = Tracer::now();
@@ -309,6 +331,15 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 p.t += p.n;
                 if (p.t < sched.end) first_of_item(p);
             };
+            // Interior tiles of a 3x3 layer (nine in ten) take a short form of the copy: every entry exists, so
+            // its address is the tile's origin (the source pixel one row and one column before the tile's
+            // first, this thread's channels) plus an offset that depends on the thread only.
+            const uint32_t pixbytes = (uint32_t)a.Cin * ESZ;
+            const uint32_t halo_off = ((uint32_t)a.Ws + 1u) * pixbytes;
+            uint32_t goffp[BATCH];
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) goffp[u] = (uint32_t)(goff[u] + (int)halo_off);
+            const char* x_thread = (const char*)a.x + j * 16;
             const uint32_t st_lo = smem_u32(smem_stage) + (uint32_t)ptid * 16u;           // + u * NUM_PRODUCERS * 16
             const uint32_t st_hi = st_lo + (uint32_t)(ITEMS * 16);
             // starts the copies of unit p; returns which of this thread's entries exist
@@ -320,6 +351,22 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 if (p.cnt == 0) { cp_async_commit(); return 0u; }  // no tile of this CTA in the item: nothing to copy
                 uint32_t vm = 7u;
                 const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
+                if (interior && !centre_only) {
+                    const uint32_t pix = ((uint32_t)tile.b * a.Hs + (uint32_t)(tile.ty0 >> up)) * a.Ws + (uint32_t)(tile.tx0 >> up);
+                    const char* org = x_thread + ((size_t)pix * pixbytes - halo_off) + (uint32_t)(c0 * ESZ);
+                    auto copy = [&](auto uc) {
+                        constexpr int u = decltype(uc)::value;
+                        const char* src = org + goffp[u];
+                        cp_async16_at<u * NUM_PRODUCERS * 16, 0>(st_lo, src);
+                        if (!IN_BF16) cp_async16_at<u * NUM_PRODUCERS * 16, 128>(st_hi, src);
+                    };
+                    copy(std::integral_constant<int, 0>{});
+                    copy(std::integral_constant<int, 1>{});
+                    copy(std::integral_constant<int, 2>{});
+                    static_assert(BATCH == 3, "one copy call per entry");
+                    cp_async_commit();
+                    return 7u;
+                }
                 if (!interior || centre_only) {
                     vm = 0u;
 #pragma unroll
@@ -603,7 +650,10 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             // store of a [4 rows x 8 pixels x slice] box; the store clips the ragged image edge.
             constexpr int NP = BN / 32;                       // 32-column passes per tile
             constexpr int PPS = OUT_MODE == 1 ? 2 : 1;        // passes per 128-byte slice
-            uint8_t* wout = smem_out + ew * (2 * WARP_SLICE_BYTES);         // this warp's two slice buffers
+            // One slice buffer per warp: before it is rewritten the warp waits until the store of the slice
+            // before has read it out.  That wait is short against an item's MMAs, the epilogue is off the
+            // critical path (two accumulator sets), and the shared memory saved is one more weight stage.
+            uint8_t* wout = smem_out + ew * (Cfg::OUT_BUFS * WARP_SLICE_BYTES);
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
             int bias_n0 = -1;
             constexpr int TAIL_BUFS = Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) >= 2 ? Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) : 2;
@@ -646,11 +696,11 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         // The CTA's last item has the weight stages to itself (every MMA has completed): its slices go
                         // through a longer ring of buffers there, so the stores of the tail are not paced by buffer reuse.
                         uint8_t* obuf = last_item ? smem_b + (ew * TAIL_BUFS + (int)((n_slice + sl) % TAIL_BUFS)) * WARP_SLICE_BYTES
-                                                  : wout + ((n_slice + sl) & 1) * WARP_SLICE_BYTES;
+                                                  : wout + (int)((n_slice + sl) % Cfg::OUT_BUFS) * WARP_SLICE_BYTES;
                         if (h == 0) {
                             if (lane == 0) {                              // the store that last read this buffer is done
                                 if (last_item) bulk_wait_group_read<TAIL_BUFS - 1>();
-                                else bulk_wait_group_read<1>();
+                                else bulk_wait_group_read<Cfg::OUT_BUFS - 1>();
                             }
                             __syncwarp();
                         }
@@ -835,6 +885,16 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 if (CG == 2) umma2_bf16_split(d, alo, a_hi, blo, b_hi, idesc, accum);
                 else umma_bf16_split(d, alo, a_hi, blo, b_hi, idesc, accum);
             };
+            // the same, predicated on the elected lane (no branch: see umma_bf16_split_on)
+            const uint32_t lead = leader ? 1u : 0u;
+            auto mma_on = [&](uint32_t d, uint32_t alo, uint32_t blo, uint32_t accum) {
+                if (CG == 2) umma2_bf16_split_on(d, alo, a_hi, blo, b_hi, idesc, accum, lead);
+                else umma_bf16_split_on(d, alo, a_hi, blo, b_hi, idesc, accum, lead);
+            };
+            auto commit_on = [&](uint32_t bar) {
+                if (CG == 2) umma2_commit_both_on(bar, lead);
+                else umma_commit_on(bar, lead);
+            };
             auto commit = [&](uint64_t* b) {
                 if (CG == 2) umma2_commit_both(smem_u32(b));
                 else umma_commit(smem_u32(b));
@@ -845,6 +905,84 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
             bool ok = true;
             int n_item = 0;
+            // Where a tap's four (eight) MMAs take 512 tensor cycles, the issuing warp has about 100 cycles
+            // to spare per tap (measured in isolation: wait + 8 MMAs + commit cost about 400), and none at
+            // the chunk and item boundaries.  So the common form (one issuing warp, one weight stage per
+            // commit; this CTA always has a tile then) runs a loop of its own: no votes (a wait that gave
+            // up leaves garbage behind that nobody reads; the abort flag is looked at once per item), the
+            // three taps of a kernel row unrolled so that their operand offsets are immediates, and every
+            // running index an addition in uniform registers.
+            constexpr bool FAST = Cfg::B_GROUP == 1 && NMMA == 1;
+            if constexpr (FAST) {
+                const uint32_t b_full0 = smem_u32(&bars->b_full[0]), b_empty0 = smem_u32(&bars->b_empty[0]);
+                auto wait_on = [&](uint32_t bar, uint32_t ph) {
+                    if (!mbar_try_wait(bar, ph)) (void)mbar_wait(bar, ph, abort_flag);
+                    tc_fence_after();
+                };
+                // one tap: its weight stage, the MMAs of the item's tile(s), the stage handed back
+                auto tap_step = [&](auto two_c, uint32_t td, uint32_t a_lo, uint32_t acc0) {
+                    constexpr bool TWO = decltype(two_c)::value;
+                    tr.mark_fine(25);
+                    wait_on(b_full0 + bs * 8u, bph);
+                    tr.mark_fine(24);
+                    const uint32_t b_lo = b_lo0 + bs * (uint32_t)(Cfg::B_STAGE_BYTES >> 4);
+                    mma_on(td, a_lo, b_lo, acc0);
+                    mma_on(td, a_lo + 2, b_lo + 2, 1u);
+                    mma_on(td, a_lo + 4, b_lo + 4, 1u);
+                    mma_on(td, a_lo + 6, b_lo + 6, 1u);
+                    if (TWO) {
+                        const uint32_t td2 = td + Cfg::ACC_COLS, a2 = a_lo + (A_TILE_BYTES >> 4);
+                        mma_on(td2, a2, b_lo, acc0);
+                        mma_on(td2, a2 + 2, b_lo + 2, 1u);
+                        mma_on(td2, a2 + 4, b_lo + 4, 1u);
+                        mma_on(td2, a2 + 6, b_lo + 6, 1u);
+                    }
+                    commit_on(b_empty0 + bs * 8u);
+                    __syncwarp();
+                    if (++bs == (uint32_t)Cfg::B_STAGES) { bs = 0; bph ^= 1; }
+                };
+                auto item = [&](auto two_c, uint32_t td, int buf) {
+                    uint32_t acc = 0;                         // the first MMA of an item overwrites the accumulator
+#pragma unroll 1
+                    for (int kc = 0; kc < ktotal; ++kc) {
+                        const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
+                        tr.mark(22);
+                        wait_on(smem_u32(&bars->a_full[as]), aph);
+                        tr.mark(23);
+                        uint32_t a_row = a_lo0 + as * (A_STAGE_BYTES >> 4);
+                        if (!centre) {
+#pragma unroll 1
+                            for (int ky = 0; ky < 3; ++ky) {
+                                tap_step(two_c, td, a_row, acc);
+                                tap_step(two_c, td, a_row + 8, 1u);
+                                tap_step(two_c, td, a_row + 16, 1u);
+                                acc = 1u;
+                                a_row += PW * 8;
+                            }
+                        } else {
+                            tap_step(two_c, td, a_row + (PW + 1) * 8, acc);
+                            acc = 1u;
+                        }
+                        commit_on(smem_u32(&bars->a_empty[as]));
+                        __syncwarp();
+                        if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
+                    }
+                    commit_on(smem_u32(&bars->acc_full[buf]));
+                    __syncwarp();
+                };
+                for (int t = sched.begin; t < sched.end; ++n_item) {
+                    const int n = sched.count(t);
+                    const int buf = n_item % NBUF;
+                    tr.mark(20);
+                    wait_on(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1);
+                    if (*abort_flag) break;
+                    tr.mark(21);
+                    const uint32_t td = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
+                    if (PAIR == 2 && sched.mine(n) == 2) item(std::true_type{}, td, buf);
+                    else item(std::false_type{}, td, buf);
+                    t += n;
+                }
+            } else
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int n = sched.count(t);
                 const int cnt = sched.mine(n);
@@ -907,6 +1045,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         else mbar_arrive(smem_u32(&bars->a_empty[as]));
                     }
                     __syncwarp();
+                    tr.mark_fine(28);
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
                 if (ok && leader) {
@@ -965,7 +1104,11 @@ EncodeTiledFn get_encode_fn() {
 }
 
 int padded_cout(int Cout) { return (Cout % 128 == 0) ? Cout : 16; }
-int pick_bn(int Cout) { return (Cout % 128 != 0) ? 16 : ((Cout % 256 == 0) ? 256 : 128); }
+int pick_bn(int Cout) {
+    static const char* e = getenv("VD_CONV_BN");     // timing studies: 128 = narrow blocks everywhere
+    if (e && e[0] == '1' && Cout % 128 == 0) return 128;
+    return (Cout % 128 != 0) ? 16 : ((Cout % 256 == 0) ? 256 : 128);
+}
 
 bool encode_weights(CUtensorMap* tm, const void* w, int Cin, int rows, int bn) {
     EncodeTiledFn enc = get_encode_fn();

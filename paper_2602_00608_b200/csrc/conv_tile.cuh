@@ -59,9 +59,6 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     return r;
 }
 __device__ __forceinline__ void load_raw_at(bool is_bf16, const char* p, Raw8& r) {
-#ifdef VD_ABL_NOLOAD      // timing study: no global loads (results are wrong)
-    r.lo = make_uint4((uint32_t)(uintptr_t)p, 2u, 3u, 4u); r.hi = r.lo; return;
-#endif
     r.lo = ldg_stream(p);
     if (!is_bf16) r.hi = ldg_stream(p + 128);
 }
