@@ -230,65 +230,60 @@ attn_tc_kernel(const AttnTcParams a, const __grid_constant__ CUtensorMap tm_q, c
         }
     } else {
         // ------------------------------------------------------------ MMA issue
-        // The whole warp runs the loop and one elected lane issues: warp-uniform code keeps the
-        // descriptors in uniform registers, which makes the wait / 4 x MMA / commit sequence of a
-        // 64-channel chunk cheaper than the 256 tensor cycles it feeds.
+        // The whole warp runs the loop and the tensor instructions are predicated on one elected lane
+        // (no branch): warp-uniform code keeps the descriptors in uniform registers, which makes the
+        // wait / 4 x MMA / commit sequence of a 64-channel chunk cheaper than the 256 tensor cycles it
+        // feeds.  The waits are not voted on (a wait that gave up leaves garbage behind that nobody
+        // reads); the abort flag is looked at once per key tile.
         {
-            const bool leader = elect_one() != 0u;
+            const uint32_t lead = elect_one();
             constexpr uint32_t idesc_s = make_idesc_bf16(128, BKV);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, DV);
             const uint32_t hi = desc_hi(1024, 2);
             uint32_t qst = 0, qph = 0, vst = 0, vph = 0;
-            bool ok = true;
+            auto wait_on = [&](uint64_t* bar, uint32_t ph) {
+                const uint32_t b = smem_u32(bar);
+                if (!mbar_try_wait(b, ph)) (void)mbar_wait(b, ph, abort_flag);
+                tc_fence_after();
+            };
             auto issue_qk = [&](int j) {
                 const int buf = j & 1;
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_free[buf]), ((j >> 1) & 1) ^ 1, abort_flag));
-                if (!ok) return;
-                tc_fence_after();
+                wait_on(&bars->s_free[buf], ((j >> 1) & 1) ^ 1);
                 for (int dc = 0; dc < dchunks; ++dc) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->qk_full[qst]), qph, abort_flag));
-                    if (!ok) return;
-                    tc_fence_after();
+                    wait_on(&bars->qk_full[qst], qph);
                     const uint32_t qa = desc_lo(smem_u32(smem_qk + qst * QK_STAGE_BYTES));
                     const uint32_t ka = qa + ((BQ * DCHUNK * 2) >> 4);
-                    if (leader) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16_split(tmem + (uint32_t)(buf * 128), qa + k * 2, hi, ka + k * 2, hi, idesc_s, (dc | k) != 0 ? 1u : 0u);
-                        umma_commit(smem_u32(&bars->qk_empty[qst]));
-                    }
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16_split_on(tmem + (uint32_t)(buf * 128), qa + k * 2, hi, ka + k * 2, hi, idesc_s, (dc | k) != 0 ? 1u : 0u, lead);
+                    umma_commit_on(smem_u32(&bars->qk_empty[qst]), lead);
                     __syncwarp();
                     if (++qst == QK_STAGES) { qst = 0; qph ^= 1; }
                 }
-                if (leader) umma_commit(smem_u32(&bars->s_full[buf]));
+                umma_commit_on(smem_u32(&bars->s_full[buf]), lead);
                 __syncwarp();
             };
             auto issue_pv = [&](int j) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full), j & 1, abort_flag));
-                if (!ok) return;
-                tc_fence_after();
+                wait_on(&bars->p_full, j & 1);
                 for (int h = 0; h < 2; ++h) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->v_full[vst]), vph, abort_flag));
-                    if (!ok) return;
-                    tc_fence_after();
+                    wait_on(&bars->v_full[vst], vph);
                     const uint32_t pa = desc_lo(smem_u32(smem_p + h * (BQ * 128)));
                     const uint32_t va = desc_lo(smem_u32(smem_v + vst * V_STAGE_BYTES));
-                    if (leader) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16_split(tmem_o, pa + k * 2, hi, va + k * 2, hi, idesc_o, (j | h | k) != 0 ? 1u : 0u);
-                        umma_commit(smem_u32(&bars->v_empty[vst]));
-                    }
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16_split_on(tmem_o, pa + k * 2, hi, va + k * 2, hi, idesc_o, (j | h | k) != 0 ? 1u : 0u, lead);
+                    umma_commit_on(smem_u32(&bars->v_empty[vst]), lead);
                     __syncwarp();
                     if (++vst == V_STAGES) { vst = 0; vph ^= 1; }
                 }
-                if (leader) umma_commit(smem_u32(&bars->pv_done));
+                umma_commit_on(smem_u32(&bars->pv_done), lead);
                 __syncwarp();
             };
             issue_qk(0);
-            for (int j = 0; j < ntiles && ok; ++j) {
+            for (int j = 0; j < ntiles; ++j) {
+                if (*abort_flag) break;
                 if (j + 1 < ntiles) issue_qk(j + 1);
-                if (ok) issue_pv(j);
+                issue_pv(j);
             }
         }
     }
