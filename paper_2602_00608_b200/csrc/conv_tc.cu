@@ -109,23 +109,30 @@ struct Bars {                    // lives in shared memory
 //
 // Two-CTA form: the range belongs to the cluster, an item is up to two tiles of one channel block,
 // and CTA `rank` of the pair takes tile t + rank (the peer has none in an odd tail item).
+//
+// Every role decodes tile numbers once per item, the fifteen producer warps among them, so the three
+// divisions are multiplications by a reciprocal the launcher computed: floor(t / d) = umulhi(t, ceil(2^32 / d)),
+// exact while t * d < 2^32 (the launcher checks it).
 struct Sched {
     int tiles_x, tiles, nblk, total;
     int begin, end, pair;
     int cg, rank;
+    uint32_t m_tiles, m_nblk, m_tx;
+    static __device__ __forceinline__ int fdiv(int t, uint32_t m) { return m ? (int)__umulhi((uint32_t)t, m) : t; }
     __device__ __forceinline__ Tile get(int t, int bn) const {
         Tile r;
-        const int blk = t / tiles;               // frame * nblk + channel block
+        const int blk = fdiv(t, m_tiles);        // frame * nblk + channel block
         const int s = t - blk * tiles;
-        r.b = blk / nblk;
+        r.b = fdiv(blk, m_nblk);
         r.n0 = (blk - r.b * nblk) * bn;
-        r.ty0 = (s / tiles_x) * TILE_H;
-        r.tx0 = (s % tiles_x) * TILE_W;
+        const int row = fdiv(s, m_tx);
+        r.ty0 = row * TILE_H;
+        r.tx0 = (s - row * tiles_x) * TILE_W;
         return r;
     }
     // number of tiles of the item that starts at tile t
     __device__ __forceinline__ int count(int t) const {
-        return ((pair == 2 || cg == 2) && t + 1 < end && (t + 1) / tiles == t / tiles) ? 2 : 1;
+        return ((pair == 2 || cg == 2) && t + 1 < end && fdiv(t + 1, m_tiles) == fdiv(t, m_tiles)) ? 2 : 1;
     }
     // of those, the tiles this CTA works on, and the s-th of them
     __device__ __forceinline__ int mine(int n) const { return cg == 2 ? (rank < n ? 1 : 0) : n; }
@@ -230,8 +237,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     // work is divided among the CTAs (CG = 1) or among the clusters of two (CG = 2)
     const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;  // 0 = leader (issues the MMAs), 1 = peer
     const int nworkers = (int)gridDim.x / CG, worker = (int)blockIdx.x / CG;
-    sched.begin = (int)(((long long)sched.total * worker) / nworkers);
-    sched.end = (int)(((long long)sched.total * (worker + 1)) / nworkers);
+    sched.begin = (int)((uint32_t)sched.total * (uint32_t)worker / (uint32_t)nworkers);          // the launcher checked the range
+    sched.end = (int)((uint32_t)sched.total * (uint32_t)(worker + 1) / (uint32_t)nworkers);
+    sched.m_tiles = a.div_tiles; sched.m_nblk = a.div_nblk; sched.m_tx = a.div_tx;
     sched.pair = PAIR;
     sched.cg = CG;
     sched.rank = (int)rank;
@@ -1170,6 +1178,15 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     else grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
     static const int grid_cap = getenv("VD_CONV_GRID") ? atoi(getenv("VD_CONV_GRID")) : 0;                      // timing studies
     if (grid_cap > 0) grid = std::max(CG, std::min(grid, grid_cap / CG * CG));
+    // reciprocals for the kernel's tile numbering (see Sched)
+    ConvArgs ka = a;
+    {
+        const int tiles_x = (a.W + TILE_W - 1) / TILE_W, nblk = padded_cout(a.Cout) / BN;
+        const int dmax = std::max(tiles, std::max(tiles_x, nblk));
+        if ((unsigned long long)total * (unsigned long long)std::max(dmax, grid + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
+        auto recip = [](int d) { return d == 1 ? 0u : (unsigned int)(((1ull << 32) + (unsigned long long)d - 1) / (unsigned long long)d); };
+        ka.div_tiles = recip(tiles); ka.div_nblk = recip(nblk); ka.div_tx = recip(tiles_x);
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -1189,7 +1206,7 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    return cudaLaunchKernelEx(&cfg, kern, a, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
+    return cudaLaunchKernelEx(&cfg, kern, ka, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
                               *(const CUtensorMap*)plan.tmap_y, status);
 }
 

@@ -29,6 +29,9 @@ struct ConvArgs {
     const float* bias2;     // [Cout] or null
     int Cin2;
     unsigned long long* trace;  // debug: per-CTA role timelines (null in production)
+    // tensor-core kernel: ceil(2^32 / d) for the divisors of its tile numbering (tiles per image, channel
+    // blocks, tiles per row), filled in by its launcher; 0 stands for d = 1
+    unsigned int div_tiles, div_nblk, div_tx;
 };
 constexpr int kConvTraceEvents = 2048;    // per (CTA, role)
 constexpr int kConvMaxCtas = 160;         // upper bound on the persistent grid (sizes the debug trace)
