@@ -210,6 +210,7 @@ class Planner {
                           ptr<void>(attno_), act_dtype(), 0, H * W, C, 3 * C, C, 1.0f / sqrtf((float)C), ptr<void>(vt_)};
         s.use_tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && attn_tc_supported(s.attn);
         fill_info(s, p + ".core", s.use_tc, C, C, 0, 0, H, W, C, act_dtype(), 0, (long)attno_);
+        if (s.use_tc) s.info.launches = 2;               // V transpose + attention core
         const double T = (double)H * W;
         s.info.flops_per_frame = 4.0 * T * T * C;
         s.info.bytes_per_frame = 4.0 * T * C * es;
