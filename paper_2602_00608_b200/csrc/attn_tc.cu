@@ -22,7 +22,7 @@ namespace {
 using namespace tc;
 
 constexpr int BQ = 128, BKV = 128, DV = 256, DCHUNK = 64;
-constexpr int QK_STAGES = 3, V_STAGES = 2;
+constexpr int QK_STAGES = 4, V_STAGES = 2;                   // as many Q/K stages as fit: the score product waits on this stream
 constexpr int QK_STAGE_BYTES = 2 * BQ * DCHUNK * 2;          // Q chunk + K chunk: 16 KB + 16 KB
 constexpr int V_STAGE_BYTES = DV * 64 * 2;                   // 256 channels x 64 keys: 32 KB
 constexpr int P_BYTES = BQ * BKV * 2;                        // 32 KB (two 64-key halves)
