@@ -151,49 +151,58 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    int tpg = 16;                                    // lanes cooperating on one group (a power of two)
-    while (tpg * a.G > kGnThreads && tpg > 1) tpg >>= 1;
-    const int sub = threadIdx.x % tpg;
-    const float inv_n = 1.f / ((float)a.P * (float)cpg);
-    for (int g0 = 0; g0 < a.G; g0 += kGnThreads / tpg) {        // uniform trip count: every lane reaches the shuffles
-        const bool valid = g0 + threadIdx.x / tpg < a.G;
-        const int g = valid ? g0 + threadIdx.x / tpg : a.G - 1;
-        const int nrec = valid ? chunks : 0;
+    // Thread t adds the records k = t / G, t / G + slices, ... of group t % G (a warp reads whole records:
+    // coalesced), the slices are added in a fixed order through shared memory, and every thread then writes
+    // scale and shift of the channels c = t, t + 512, ...
+    const int slices = kGnThreads / a.G;             // >= 1 (checked by the launcher)
+    const int g = threadIdx.x % a.G, sl = threadIdx.x / a.G;
+    float2 acc = make_float2(0.f, 0.f);
+    if (sl < slices) {
         const float2* rec = (const float2*)a.partial + (size_t)n * kGnMaxChunks * a.G + g;
-        // loads that do not depend on the records go first, so one memory round trip covers them all
-        float kv[4];
-        load4<T>(x + (size_t)(a.P / 2) * a.C + g * cpg, kv);
-        const int c0 = g * cpg + min(sub, cpg - 1);
-        const float gamma0 = __ldg(a.gamma + c0), beta0 = __ldg(a.beta + c0);
-        float2 acc = make_float2(0.f, 0.f);
-        for (int k0 = sub; k0 < nrec; k0 += kGnFinalLoads * tpg) {
+        for (int k0 = sl; k0 < chunks; k0 += kGnFinalLoads * slices) {
             float2 r[kGnFinalLoads];
+            // unconditional loads (a record that does not exist re-reads the first and counts as zero), issued
+            // back to back before the first use
 #pragma unroll
             for (int i = 0; i < kGnFinalLoads; ++i) {
-                const int k = k0 + i * tpg;
-                r[i] = (k < nrec) ? __ldcg(rec + (size_t)k * a.G) : make_float2(0.f, 0.f);
+                const int k = k0 + i * slices;
+                const float2* q = rec + (size_t)(k < chunks ? k : sl) * a.G;
+                asm volatile("ld.global.cg.v2.f32 {%0, %1}, [%2];" : "=f"(r[i].x), "=f"(r[i].y) : "l"(q));
             }
 #pragma unroll
             for (int i = 0; i < kGnFinalLoads; ++i) {
-                acc.x += r[i].x;
-                acc.y += r[i].y;
+                const bool on = k0 + i * slices < chunks;
+                acc.x += on ? r[i].x : 0.f;
+                acc.y += on ? r[i].y : 0.f;
             }
         }
-        for (int d = tpg >> 1; d > 0; d >>= 1) {     // a + b == b + a: both lanes of a pair end with equal values
-            acc.x += __shfl_xor_sync(0xffffffffu, acc.x, d);
-            acc.y += __shfl_xor_sync(0xffffffffu, acc.y, d);
+    }
+    __syncthreads();                                 // the block's own use of sm[] above is over
+    sm[threadIdx.x] = acc;
+    __syncthreads();
+    __shared__ float s_mean[kGnThreads], s_rstd[kGnThreads];
+    if (threadIdx.x < a.G) {
+        float2 t = make_float2(0.f, 0.f);
+        for (int q = 0; q < slices; ++q) {
+            const float2 v = sm[q * a.G + threadIdx.x];
+            t.x += v.x;
+            t.y += v.y;
         }
+        float kv[4];
+        load4<T>(x + (size_t)(a.P / 2) * a.C + threadIdx.x * cpg, kv);
         const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
-        const float md = acc.x * inv_n;
-        const float var = fmaxf(fmaf(-md, md, acc.y * inv_n), 0.f);
-        const float mean = k + md;
-        const float rstd = 1.f / sqrtf(var + a.eps);
-        for (int cc = sub; valid && cc < cpg; cc += tpg) {
-            const int c = g * cpg + cc;
-            const float sc = (cc == sub ? gamma0 : a.gamma[c]) * rstd;
-            a.scale[(size_t)n * a.C + c] = sc;
-            a.shift[(size_t)n * a.C + c] = (cc == sub ? beta0 : a.beta[c]) - mean * sc;
-        }
+        const float inv_n = 1.f / ((float)a.P * (float)cpg);
+        const float md = t.x * inv_n;
+        const float var = fmaxf(fmaf(-md, md, t.y * inv_n), 0.f);
+        s_mean[threadIdx.x] = k + md;
+        s_rstd[threadIdx.x] = 1.f / sqrtf(var + a.eps);
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < a.C; c += kGnThreads) {
+        const int gc = c / cpg;
+        const float sc = __ldg(a.gamma + c) * s_rstd[gc];
+        a.scale[(size_t)n * a.C + c] = sc;
+        a.shift[(size_t)n * a.C + c] = __ldg(a.beta + c) - s_mean[gc] * sc;
     }
     if (threadIdx.x == 0) a.counters[n] = 0u;        // ready for the next launch
 }
