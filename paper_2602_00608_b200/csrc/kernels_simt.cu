@@ -76,7 +76,7 @@ template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bflo
 }
 
 constexpr int kGnThreads = 512;
-constexpr int kGnFinalLoads = (kGnMaxChunks + 15) / 16;   // records per lane when 16 lanes share a group
+constexpr int kGnFinalLoads = (kGnMaxChunks + 15) / 16;   // records a thread of the last block reads in one round (32 groups: 16 slices)
 
 template <typename T, int U>
 __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int chunks, int pix_per_chunk) {
