@@ -15,6 +15,7 @@ VD_OK, VD_ERR_INVALID_ARG, VD_ERR_UNSUPPORTED, VD_ERR_WORKSPACE, VD_ERR_CUDA, VD
 VD_F32, VD_BF16 = 0, 1
 VD_ARCH_TINY, VD_ARCH_SDVAE = 0, 1
 VD_FLAG_FORCE_SIMT = 0x1
+VD_FLAG_UPSAMPLE_9TAP = 0x2
 VD_IMPL_AUTO, VD_IMPL_SIMT, VD_IMPL_TC = 0, 1, 2
 VD_STEP_INGEST, VD_STEP_GN_STATS, VD_STEP_CONV, VD_STEP_ATTENTION = 0, 1, 2, 3
 STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", -3: "VD_ERR_WORKSPACE",
@@ -24,7 +25,7 @@ EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
     "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
-    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_debug_conv_trace",
+    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_debug_status_offset", "vd_debug_wait_probe",
 ]
 
 
@@ -44,7 +45,7 @@ class VdStepInfo(Structure):
                 ("out_h", c_int32), ("out_w", c_int32), ("out_channels", c_int32), ("out_dtype", c_int32),
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
                 ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
-                ("has_residual", c_int32), ("reserved", c_int32 * 2)]
+                ("has_residual", c_int32), ("phase_collapsed", c_int32), ("reserved", c_int32 * 1)]
 
 
 class VdConvDesc(Structure):
@@ -84,7 +85,9 @@ def lib():
         l.vd_get_step.argtypes = [vp, c_int32, POINTER(VdStepInfo)]
         l.vd_profile.argtypes = [vp, vp, vp, c_int32, vp, POINTER(c_float), c_int32]
         l.vd_debug_stop_after.argtypes = [vp, c_int32]
-        l.vd_debug_conv_trace.argtypes = [vp, c_size_t]
+        l.vd_clear_status.argtypes = [vp, vp]
+        l.vd_debug_status_offset.argtypes = [vp, POINTER(c_int64)]
+        l.vd_debug_wait_probe.argtypes = [vp, c_int64, vp]
         l.vd_conv_packed_weight_bytes.argtypes = [POINTER(VdConvDesc), POINTER(c_size_t)]
         l.vd_conv_pack_weight.argtypes = [POINTER(VdConvDesc), vp, c_int32, vp, vp]
         l.vd_op_conv2d.argtypes = [POINTER(VdConvDesc), vp, vp, vp, vp, vp, vp, vp, vp]
@@ -206,6 +209,18 @@ class Decoder:
     # ---- introspection
     def check_status(self):
         _check(lib().vd_get_status(self.handle), self.handle)
+
+    def clear_status(self, stream=None):
+        _check(lib().vd_clear_status(self.handle, _stream_ptr(stream)), self.handle)
+
+    def status_word(self):
+        """The four 32-bit words of the device status record, as a view of the workspace (for tests)."""
+        off = c_int64(0)
+        _check(lib().vd_debug_status_offset(self.handle, byref(off)), self.handle)
+        return self.workspace[off.value: off.value + 16].view(self.torch.int32)
+
+    def wait_probe(self, limit_cycles: int, stream=None):
+        _check(lib().vd_debug_wait_probe(self.handle, limit_cycles, _stream_ptr(stream)), self.handle)
 
     def steps(self):
         n = c_int32(0)

@@ -11,9 +11,9 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libvd.so")
-SOURCES = ["vd_api.cu", "kernels_simt.cu", "conv_tc.cu", "attn_tc.cu"]
+SOURCES = ["vd_api.cu", "kernels_simt.cu", "conv_tc.cu", "attn_tc.cu", "wait_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC,-fvisibility=hidden", "--use_fast_math" if False else "-DVD_BUILD",
+              "-Xcompiler", "-fPIC,-fvisibility=hidden", "-DVD_BUILD",
               "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 

@@ -291,7 +291,7 @@ attn_tc_kernel(const AttnTcParams a, const __grid_constant__ CUtensorMap tm_q, c
     tc_fence_before();
     __syncthreads();
     if (tid == 0 && bars->abort_flag && status) {
-        if (atomicCAS(status, 0u, 0xC0DE0002u) == 0u) {
+        if (atomicCAS(status, 0u, kStatusAttnTimeout) == 0u) {
             status[1] = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
             status[2] = 0;
         }

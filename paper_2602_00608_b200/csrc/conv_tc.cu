@@ -38,6 +38,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <type_traits>
 
 #include "conv_tile.cuh"
@@ -52,11 +53,6 @@ using namespace tc;
 using namespace convtile;
 
 constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
-// MMA-issuing warps for two-tile items: one warp issuing for both tiles measures 2 % faster than one warp per
-// tile now that the issue loop is warp-uniform (the two-warp form stays selectable for timing studies)
-#ifndef VD_NMMA
-#define VD_NMMA 1
-#endif
 constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epilogue warp's share of an output slice
 
 // BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
@@ -71,13 +67,26 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // that gate the MMAs live in the leader: the peer's producers and weight loads signal the leader's
 // "full" barriers across the cluster, its epilogue the leader's "accumulator free" barrier, and the
 // leader's tcgen05.commit arrives on the "empty" / "accumulator ready" barriers of both CTAs.
-template <int BN, int CG = 1> struct TileCfg {
-    static_assert(CG == 1 || BN == 256, "the two-CTA form exists for 256-channel blocks only");
-    static constexpr int PAIR = BN == 256 ? 1 : 2;                   // tiles per work item (and CTA)
-    static constexpr int B_STAGE_BYTES = (BN / CG) * 128;            // this CTA's rows x 64 bf16
-    static constexpr int OUT_BUFS = 1;                               // output slices per epilogue warp
+//
+// PH (phase-collapsed nearest-2x upsampling + 3x3, BN = 128 on CTA pairs): a 3x3 convolution of the
+// upsampled tensor is, for each of the four output parities (a, b) = (row & 1, column & 1), a 2x2
+// convolution of the SOURCE tensor whose weights are sums of the 3x3 taps that fall on the same source
+// pixel (rows: parity 0 reads source rows {i-1 <- ky 0; i <- ky 1+2}, parity 1 {i <- ky 0+1; i+1 <- ky 2};
+// columns alike).  So the tile is 16x8 SOURCE pixels, its one halo tile feeds four accumulators
+// (one per parity, 128 columns each: all of tensor memory) through 4 x 4 tap views, and 16 instead
+// of 4 x 9 = 36 tap products are issued per source pixel and 64-channel chunk: 4/9 of the work.
+// The accumulators have no second set; instead each parity has its own "full"/"empty" barriers and
+// is drained as soon as its last tap has completed, while the MMAs of the other parities go on.
+// A weight stage holds the two column taps (dx = 0, 1) of one (parity, dy): 8 MMAs per stage, so
+// the issue sequence per stage is as long as that of the other forms.
+template <int BN, int CG = 1, bool PH = false> struct TileCfg {
+    static_assert(CG == 1 || BN == 256 || PH, "the two-CTA form exists for 256-channel blocks and the phase form");
+    static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
+    static constexpr int PAIR = PH ? 1 : (BN == 256 ? 1 : 2);        // tiles per work item (and CTA)
+    static constexpr int B_STAGE_BYTES = (PH ? 2 : 1) * (BN / CG) * 128;   // this CTA's rows x 64 bf16 (phase: two taps)
+    static constexpr int OUT_BUFS = PH ? 2 : 1;                      // output slices per epilogue warp
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
-    static constexpr int B_STAGES = CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8));
+    static constexpr int B_STAGES = PH ? 5 : (CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = 2;
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
@@ -85,20 +94,20 @@ template <int BN, int CG = 1> struct TileCfg {
     static constexpr int SMEM_OUT = BN >= 128 ? OUT_BUFS * OUT_SLICE_BYTES : 0;       // output slice(s) per epilogue warp
     static constexpr int SMEM_A = A_STAGES * A_STAGE_BYTES - (A_TILE_BYTES - NPIX * 128);   // the last tile needs no padding
     static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
-    static constexpr int SMEM_BARS = 256;
+    static constexpr int SMEM_BARS = 512;
     // two-tile items and two-CTA pairs: the producers stage the raw input of the next unit in shared memory (cp.async)
     static constexpr bool STAGED = PAIR == 2 || CG == 2;
     static constexpr int SMEM_RAW = STAGED ? ITEMS * 32 : 0;
     static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + SMEM_BARS + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
-    static constexpr int NBUF = 2;                                   // accumulator sets (PAIR tiles each)
-    static constexpr int TMEM_COLS = NBUF * PAIR * ACC_COLS;
+    static constexpr int NBUF = PH ? 1 : 2;                          // accumulator sets (PAIR tiles each; phase: four parities)
+    static constexpr int TMEM_COLS = PH ? 4 * ACC_COLS : NBUF * PAIR * ACC_COLS;
 };
 
 struct Bars {                    // lives in shared memory
     uint64_t a_full[MAX_A_STAGES], a_empty[MAX_A_STAGES];
     uint64_t b_full[MAX_B_STAGES], b_empty[MAX_B_STAGES];
-    uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_full[4], acc_empty[4];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -203,13 +212,12 @@ __device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
 
 // OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC (both through shared memory and TMA stores),
 //           2 = NCHW frame written directly (dtype from a.out_dtype)
-template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1>
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, unsigned int* status) {
-    using Cfg = TileCfg<BN, CG>;
+    using Cfg = TileCfg<BN, CG, PH>;
     constexpr int NBUF = Cfg::NBUF, PAIR = Cfg::PAIR, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
-    constexpr int NMMA = PAIR == 2 ? VD_NMMA : 1;            // MMA-issuing warps
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* smem_b = smem;
@@ -222,7 +230,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     uint8_t* smem_stage = smem_bias + Cfg::SMEM_BIAS + Cfg::SMEM_BARS;  // raw input of the next unit (two-tile items only)
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
-    const long long t_entry = Tracer::now();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int taps = a.ksize * a.ksize;
     const int kchunks = a.Cin >> 6;
@@ -246,9 +253,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
 
     if (tid == 0) {
         // CG = 2: the leader's "full" barriers collect the arrivals of both CTAs; commits go to both CTAs
-        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), CG * NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), NMMA); }
-        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), CG); mbar_init(smem_u32(&bars->b_empty[i]), NMMA); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), NMMA); mbar_init(smem_u32(&bars->acc_empty[i]), 4 * CG); }
+        for (int i = 0; i < Cfg::A_STAGES; ++i) { mbar_init(smem_u32(&bars->a_full[i]), CG * NUM_PRODUCER_WARPS); mbar_init(smem_u32(&bars->a_empty[i]), 1); }
+        for (int i = 0; i < Cfg::B_STAGES; ++i) { mbar_init(smem_u32(&bars->b_full[i]), CG); mbar_init(smem_u32(&bars->b_empty[i]), 1); }
+        for (int i = 0; i < 4; ++i) { mbar_init(smem_u32(&bars->acc_full[i]), 1); mbar_init(smem_u32(&bars->acc_empty[i]), 4 * CG); }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -304,7 +311,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const bool inner = py >= 1 && py <= TILE_H && px >= 1 && px <= TILE_W;
             pyx[u] = (uint32_t)py | ((uint32_t)px << 8) | (inner ? 1u << 16 : 0u);
         }
-        Tracer tr; tr.init(ptid == 0 ? a.trace : nullptr, 0);
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         griddep_wait();              // everything above is arithmetic on the thread's own indices
@@ -442,7 +448,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const bool in_bf16 = IN_BF16 && !second;
                 advance(nx);
                 const bool have_next = nx.t < sched.end;
-                tr.mark(1);
                 cp_async_wait_all();                             // this thread's pieces of the current unit have landed
                 Raw8 raw[BATCH];
 #pragma unroll
@@ -455,7 +460,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                     if (!ok) break;
                 }
-                tr.mark(2);
                 uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur_slot * A_TILE_BYTES;
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
@@ -493,7 +497,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     if (++stage == Cfg::A_STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (have_next && (nx.kc != cur_kc || nx.t != cur_t)) load_affine(nx);
-                tr.mark(3);
                 have = have_next;
             }
             cp_async_wait_all();
@@ -531,7 +534,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             tile.tx0 += TILE_W;
                             if (tile.tx0 >= sched.tiles_x * TILE_W) { tile.tx0 = 0; tile.ty0 += TILE_H; }
                         }
-                        tr.mark(1);
                         // which entries exist: all of them where the halo lies inside the image
                         uint32_t vm = 7u;
                         const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
@@ -564,7 +566,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                             if (!ok) break;
                         }
-                        tr.mark(2);
                         uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + slot * A_TILE_BYTES;
                         const bool in_bf16 = IN_BF16 && !second;
 #pragma unroll
@@ -596,7 +597,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
                             }
                         }
-                        tr.mark(3);
                     }
                 }
                 if (!ok) break;
@@ -615,7 +615,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         griddep_wait();
         const int ew = warp - EPI_WARP0;                     // TMEM lane quarter
         const bool reduce_add = a.residual != nullptr;       // y is the residual stream: the tile is added into it
-        Tracer tr; tr.init(tid == EPI_WARP0 * 32 ? a.trace : nullptr, 2);
         bool ok = true;
         int n_item = 0;
         uint32_t n_slice = 0;
@@ -669,20 +668,34 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const int n = sched.count(t);
                 const int cnt = sched.mine(n);
                 const int buf = n_item % NBUF;
-                const bool last_item = t + n >= sched.end && Cfg::SMEM_B >= 8 * WARP_SLICE_BYTES;
-                tr.mark(10);
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                tr.mark(11);
-                if (cnt == 0) {                              // nothing of this CTA in the accumulators: hand them back at once
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) arrive_leader(&bars->acc_empty[buf]);
+                // (phase form: the weight stages stay in use while the first parities are drained)
+                const bool last_item = !PH && t + n >= sched.end && Cfg::SMEM_B >= 8 * WARP_SLICE_BYTES;
+                if (!PH) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[buf]), (n_item / NBUF) & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (cnt == 0) {                          // nothing of this CTA in the accumulators: hand them back at once
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_leader(&bars->acc_empty[buf]);
+                    }
                 }
+                // sub-tiles of the item: its tiles, or (phase form) the four output parities of its one source tile
+                const int nsub = PH ? 4 : cnt;
 #pragma unroll 1
-                for (int slot = 0; slot < cnt; ++slot) {
-                    const Tile tl = sched.get(sched.index(t, slot), BN);
+                for (int slot = 0; slot < nsub; ++slot) {
+                    if (PH) {                                // parity `slot` is complete once its last tap has been committed
+                        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_full[slot]), n_item & 1, abort_flag));
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (cnt == 0) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) arrive_leader(&bars->acc_empty[slot]);
+                            continue;
+                        }
+                    }
+                    const Tile tl = sched.get(sched.index(t, PH ? 0 : slot), BN);
                     if (tl.n0 != bias_n0) {                   // (re)load bias (+ shortcut bias) of this channel block
                         __syncwarp();
                         for (int i = lane; i < BN; i += 32)
@@ -691,7 +704,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         __syncwarp();
                     }
                     const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
-                    const bool last_tile = slot == cnt - 1;
+                    const bool last_tile = PH || slot == cnt - 1;
+                    const int acc_bar = PH ? slot : buf;
                     uint32_t ra[32], rb[32];
                     tmem_ld32(tacc, ra);
                     tmem_ld_wait();
@@ -738,14 +752,17 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         } else if (last_tile) {                          // accumulators fully read: hand them back
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) arrive_leader(&bars->acc_empty[buf]);
+                            if (lane == 0) arrive_leader(&bars->acc_empty[acc_bar]);
                         }
                         if (h == PPS - 1) {
                             fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) {
                                 constexpr int CS = 32 * PPS;
-                                if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
+                                // phase form: the tile is one parity of a 32x16 output block: rows 2i + a through the map of
+                                // row parity a (tmap_y, tmap2), columns 2j + b through the map's parity coordinate
+                                if (PH) tma_store_5d((slot >> 1) ? &tmap2 : &tmap_y, smem_u32(obuf), tl.n0 + sl * CS, slot & 1, tl.tx0, tl.ty0 + 4 * ew, tl.b);
+                                else if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
                                 else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
                                 bulk_commit_group();
                             }
@@ -756,7 +773,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 t += n;
             }
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
-            tr.mark(12);
         }
     } else if (warp == PREFETCH_WARP) {
         // ------------------------------------------------ input prefetch into L2
@@ -827,21 +843,36 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)
         if (lane == 0) {
-            Tracer tr; tr.init(a.trace, 3);
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
             for (int t = sched.begin; t < sched.end && ok; t += sched.count(t)) {
                 const Tile tl = sched.get(t, BN);
+                if constexpr (PH) {
+                    // eight stages per chunk: (parity, dy), each with the taps dx = 0, 1 of this CTA's 64 output
+                    // channels as one box of 128 rows (the packed layout keeps them adjacent)
+                    const int blk = tl.n0 / BN;
+                    for (int kc = 0; kc < kchunks && ok; ++kc) {
+                        for (int st = 0; st < 8; ++st) {
+                            ok = mbar_wait(smem_u32(&bars->b_empty[stage]), phase ^ 1, abort_flag);
+                            if (!ok) break;
+                            const uint32_t dst = smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES);
+                            const uint32_t full = leader_bar(&bars->b_full[stage]);
+                            mbar_arrive_expect_tx_cluster(full, Cfg::B_STAGE_BYTES);
+                            tma_load_2d_pair(dst, &tmap, kc * 64, ((st * sched.nblk + blk) * 2 + (int)rank) * 128, full);
+                            ++issued;
+                            if (++stage == Cfg::B_STAGES) { stage = 0; phase ^= 1; }
+                        }
+                    }
+                    continue;
+                }
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
                     for (int tap = 0; tap < ntap; ++tap) {
                         if (stage % Cfg::B_GROUP == 0) {     // stages come back in groups (see the MMA thread)
-                            tr.mark(30);
                             ok = mbar_wait(smem_u32(&bars->b_empty[stage / Cfg::B_GROUP]), phase ^ 1, abort_flag);
                             if (!ok) break;
-                            tr.mark(31);
                         }
                         const uint32_t dst = smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES);
                         if (CG == 2) {       // this CTA's half of the rows; completion is reported to the leader's barrier
@@ -872,22 +903,18 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
             }
         }
-    } else if ((warp == MMA_WARP && rank == 0) || (NMMA == 2 && warp == MMA_WARP2)) {
+    } else if (warp == MMA_WARP && rank == 0) {
         // ------------------------------------------------ MMA issue
         // The whole warp runs the loop and one elected lane issues: in warp-uniform code the
         // compiler keeps descriptors and counters in uniform registers, and the issue sequence of
         // wait / 4 x tcgen05.mma / commit costs about 300 cycles instead of about 480 from a
         // single-lane branch (measured), which a tap's 513 tensor cycles then hide.  Where an item
-        // is two tiles the warp issues for both (VD_NMMA = 2 gives each tile its own issuing warp:
-        // both then follow every barrier in lockstep and both arrive on the "empty"/"full" barriers
-        // they release, by tcgen05.commit when they issued MMAs and plainly when an odd tail item
-        // has no second tile).
+        // is two tiles the warp issues for both.
         {
-            const int me = warp == MMA_WARP ? 0 : 1;          // the tile slot this warp issues for
             const bool leader = elect_one() != 0u;
             constexpr uint32_t idesc = make_idesc_bf16(128 * CG, BN);
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
-            const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)) + me * (A_TILE_BYTES >> 4), b_lo0 = desc_lo(smem_u32(smem_b));
+            const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)), b_lo0 = desc_lo(smem_u32(smem_b));
             // one MMA of the pair (M = 256 over both CTAs) or of this CTA; a commit to both CTAs or to this one
             auto mma = [&](uint32_t d, uint32_t alo, uint32_t blo, uint32_t accum) {
                 if (CG == 2) umma2_bf16_split(d, alo, a_hi, blo, b_hi, idesc, accum);
@@ -907,9 +934,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 if (CG == 2) umma2_commit_both(smem_u32(b));
                 else umma_commit(smem_u32(b));
             };
-            Tracer tr; tr.init((me == 0 && lane == 0) ? a.trace : nullptr, 1);
-            tr.mark_at(40, t_entry);
-            tr.mark(41);
             uint32_t as = 0, aph = 0, bs = 0, bph = 0;
             bool ok = true;
             int n_item = 0;
@@ -920,7 +944,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             // up leaves garbage behind that nobody reads; the abort flag is looked at once per item), the
             // three taps of a kernel row unrolled so that their operand offsets are immediates, and every
             // running index an addition in uniform registers.
-            constexpr bool FAST = Cfg::B_GROUP == 1 && NMMA == 1;
+            constexpr bool FAST = Cfg::B_GROUP == 1;
             if constexpr (FAST) {
                 const uint32_t b_full0 = smem_u32(&bars->b_full[0]), b_empty0 = smem_u32(&bars->b_empty[0]);
                 auto wait_on = [&](uint32_t bar, uint32_t ph) {
@@ -930,9 +954,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 // one tap: its weight stage, the MMAs of the item's tile(s), the stage handed back
                 auto tap_step = [&](auto two_c, uint32_t td, uint32_t a_lo, uint32_t acc0) {
                     constexpr bool TWO = decltype(two_c)::value;
-                    tr.mark_fine(25);
                     wait_on(b_full0 + bs * 8u, bph);
-                    tr.mark_fine(24);
                     const uint32_t b_lo = b_lo0 + bs * (uint32_t)(Cfg::B_STAGE_BYTES >> 4);
                     mma_on(td, a_lo, b_lo, acc0);
                     mma_on(td, a_lo + 2, b_lo + 2, 1u);
@@ -954,9 +976,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
 #pragma unroll 1
                     for (int kc = 0; kc < ktotal; ++kc) {
                         const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
-                        tr.mark(22);
                         wait_on(smem_u32(&bars->a_full[as]), aph);
-                        tr.mark(23);
                         uint32_t a_row = a_lo0 + as * (A_STAGE_BYTES >> 4);
                         if (!centre) {
 #pragma unroll 1
@@ -978,13 +998,58 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     commit_on(smem_u32(&bars->acc_full[buf]));
                     __syncwarp();
                 };
+                // phase form: per chunk, the four parities' 2 x 2 taps (see TileCfg); parity p = 2a + b accumulates
+                // in columns [128p, 128p + 128), waits for its own "empty" barrier before the item's first tap and
+                // reports "full" after its last, so the epilogue drains parity 0 while parities 1..3 still compute
+                auto item_phase = [&](int n_it) {
+#pragma unroll 1
+                    for (int kc = 0; kc < kchunks; ++kc) {
+                        const bool first = kc == 0, last = kc == kchunks - 1;
+                        wait_on(smem_u32(&bars->a_full[as]), aph);
+                        const uint32_t a_base = a_lo0 + as * (A_STAGE_BYTES >> 4);
+#pragma unroll
+                        for (int p = 0; p < 4; ++p) {
+                            const uint32_t td = tmem_base + (uint32_t)(p * Cfg::ACC_COLS);
+                            if (first) wait_on(smem_u32(&bars->acc_empty[p]), (uint32_t)((n_it & 1) ^ 1));
+#pragma unroll
+                            for (int dy = 0; dy < 2; ++dy) {
+                                wait_on(b_full0 + bs * 8u, bph);
+                                const uint32_t b_lo = b_lo0 + bs * (uint32_t)(Cfg::B_STAGE_BYTES >> 4);
+                                const uint32_t a_lo = a_base + (uint32_t)((((p >> 1) + dy) * PW + (p & 1)) * 8);
+                                mma_on(td, a_lo, b_lo, (first && dy == 0) ? 0u : 1u);
+                                mma_on(td, a_lo + 2, b_lo + 2, 1u);
+                                mma_on(td, a_lo + 4, b_lo + 4, 1u);
+                                mma_on(td, a_lo + 6, b_lo + 6, 1u);
+                                constexpr uint32_t B_TAP = (uint32_t)(Cfg::B_STAGE_BYTES >> 5);     // second tap of the stage
+                                mma_on(td, a_lo + 8, b_lo + B_TAP, 1u);
+                                mma_on(td, a_lo + 10, b_lo + B_TAP + 2, 1u);
+                                mma_on(td, a_lo + 12, b_lo + B_TAP + 4, 1u);
+                                mma_on(td, a_lo + 14, b_lo + B_TAP + 6, 1u);
+                                commit_on(b_empty0 + bs * 8u);
+                                __syncwarp();
+                                if (++bs == (uint32_t)Cfg::B_STAGES) { bs = 0; bph ^= 1; }
+                            }
+                            if (last) {
+                                commit_on(smem_u32(&bars->acc_full[p]));
+                                __syncwarp();
+                            }
+                        }
+                        commit_on(smem_u32(&bars->a_empty[as]));
+                        __syncwarp();
+                        if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
+                    }
+                };
                 for (int t = sched.begin; t < sched.end; ++n_item) {
                     const int n = sched.count(t);
+                    if constexpr (PH) {
+                        if (*abort_flag) break;
+                        item_phase(n_item);
+                        t += n;
+                        continue;
+                    }
                     const int buf = n_item % NBUF;
-                    tr.mark(20);
                     wait_on(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1);
                     if (*abort_flag) break;
-                    tr.mark(21);
                     const uint32_t td = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
                     if (PAIR == 2 && sched.mine(n) == 2) item(std::true_type{}, td, buf);
                     else item(std::false_type{}, td, buf);
@@ -994,34 +1059,28 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int n = sched.count(t);
                 const int cnt = sched.mine(n);
-                const bool active = me < cnt;
+                const bool active = cnt > 0;
                 const int buf = n_item % NBUF;
-                tr.mark(20);
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                tr.mark(21);
-                const uint32_t td = tmem_base + (uint32_t)((buf * PAIR + me) * Cfg::ACC_COLS);
+                const uint32_t td = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
                 uint32_t acc = 0;                             // the first MMA of an item overwrites the accumulator
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
                     const int ntap = centre ? 1 : 9;
-                    tr.mark(22);
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
-                    tr.mark(23);
                     // tap view: rows start (ky*PW + kx) pixels into the halo tile; eight-row groups are
                     // one tile row (PW pixels) apart.  The tensor core applies the 128-byte swizzle to the
                     // absolute shared-memory address, so any 128-byte-aligned start works (base_offset 0).
                     uint32_t a_lo = a_lo0 + as * (A_STAGE_BYTES >> 4) + (centre ? (PW + 1) * 8 : 0);   // + (ky*PW + kx) * 128 B >> 4
                     int kx = 0;
                     for (int tap = 0; tap < ntap; ++tap) {
-                        tr.mark_fine(25);
                         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->b_full[bs]), bph, abort_flag));
                         if (!ok) break;
                         tc_fence_after();
-                        tr.mark_fine(24);
                         const uint32_t b_lo = b_lo0 + bs * (Cfg::B_STAGE_BYTES >> 4);
                         if (leader) {
                             if (active) {
@@ -1029,7 +1088,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 mma(td, a_lo + 2, b_lo + 2, 1u);
                                 mma(td, a_lo + 4, b_lo + 4, 1u);
                                 mma(td, a_lo + 6, b_lo + 6, 1u);
-                                if (PAIR == 2 && NMMA == 1 && cnt == 2) {       // one warp issues for both tiles
+                                if (PAIR == 2 && cnt == 2) {       // one warp issues for both tiles
                                     const uint32_t td2 = td + Cfg::ACC_COLS, a2 = a_lo + (A_TILE_BYTES >> 4);
                                     mma(td2, a2, b_lo, acc);
                                     mma(td2, a2 + 2, b_lo + 2, 1u);
@@ -1053,7 +1112,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         else mbar_arrive(smem_u32(&bars->a_empty[as]));
                     }
                     __syncwarp();
-                    tr.mark_fine(28);
                     if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                 }
                 if (ok && leader) {
@@ -1070,7 +1128,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     __syncthreads();
     if (CG == 2) cluster_sync_all();                         // nobody leaves while the pair may still touch its memory
     if (tid == 0 && bars->abort_flag && status) {
-        if (atomicCAS(status, 0u, 0xC0DE0001u) == 0u) {
+        if (atomicCAS(status, 0u, kStatusConvTimeout) == 0u) {
             status[1] = blockIdx.x;
             status[2] = (uint32_t)BN;
         }
@@ -1097,6 +1155,36 @@ __global__ void pack_weight_tc_kernel(const T* w, __nv_bfloat16* packed, int Cou
     }
 }
 
+// Phase-collapsed upsampling convolution: OIHW 3x3 -> bf16 rows of Cin, ordered
+// [stage = 2 * parity + dy][128-channel block][CTA rank][dx][64 channels], parity = 2a + b, so that the two
+// column taps of one (parity, dy) for one CTA's half of a channel block are one box of 128 rows.
+// The weight at (parity (a, b), dy, dx) is the sum of the 3x3 taps (ky, kx) that read the same source
+// pixel: a = 0: dy 0 <- ky {0}, dy 1 <- ky {1, 2};  a = 1: dy 0 <- ky {0, 1}, dy 1 <- ky {2};  columns alike.
+// The sum is formed in fp32 in a fixed order and rounded once to bf16.
+template <typename T>
+__global__ void pack_weight_phase_kernel(const T* w, __nv_bfloat16* packed, int Cout, int Cin) {
+    const int64_t total = (int64_t)16 * Cout * Cin;
+    const int nblk = Cout / 128;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % Cin);
+        const int o = (int)((i / Cin) % Cout);
+        const int tap = (int)(i / ((int64_t)Cin * Cout));          // 0..15: parity * 4 + dy * 2 + dx
+        const int par = tap >> 2, dy = (tap >> 1) & 1, dx = tap & 1;
+        const int pa = par >> 1, pb = par & 1;
+        const int ky0 = pa == 0 ? (dy == 0 ? 0 : 1) : (dy == 0 ? 0 : 2), ky1 = pa == 0 ? (dy == 0 ? 0 : 2) : (dy == 0 ? 1 : 2);
+        const int kx0 = pb == 0 ? (dx == 0 ? 0 : 1) : (dx == 0 ? 0 : 2), kx1 = pb == 0 ? (dx == 0 ? 0 : 2) : (dx == 0 ? 1 : 2);
+        float v = 0.f;
+        for (int ky = ky0; ky <= ky1; ++ky)
+            for (int kx = kx0; kx <= kx1; ++kx) {
+                const size_t j = ((size_t)o * Cin + c) * 9 + ky * 3 + kx;
+                v += sizeof(T) == 2 ? __bfloat162float(((const __nv_bfloat16*)w)[j]) : ((const float*)w)[j];
+            }
+        const int st = par * 2 + dy, blk = o / 128, rk = (o % 128) / 64, r = o % 64;
+        const size_t row = ((((size_t)st * nblk + blk) * 2 + rk) * 2 + dx) * 64 + r;
+        packed[row * Cin + c] = __float2bfloat16_rn(v);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -1113,8 +1201,6 @@ EncodeTiledFn get_encode_fn() {
 
 int padded_cout(int Cout) { return (Cout % 128 == 0) ? Cout : 16; }
 int pick_bn(int Cout) {
-    static const char* e = getenv("VD_CONV_BN");     // timing studies: 128 = narrow blocks everywhere
-    if (e && e[0] == '1' && Cout % 128 == 0) return 128;
     return (Cout % 128 != 0) ? 16 : ((Cout % 256 == 0) ? 256 : 128);
 }
 
@@ -1128,15 +1214,6 @@ bool encode_weights(CUtensorMap* tm, const void* w, int Cin, int rows, int bn) {
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int num_sms() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
 }
 
 // clusters of two CTAs of this kernel that the device can hold at once (0: the form cannot run)
@@ -1156,32 +1233,54 @@ int max_pairs(K kern, int smem) {
     return n;
 }
 
-template <int BN, bool IB, int OM, int CG>
-cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM, CG>;
-    constexpr int SMEM = TileCfg<BN, CG>::SMEM_TOTAL;
-    static bool configured = false;
-    static int pairs = 0;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+// Per-device launch state of one kernel instantiation (the shared-memory attribute is per device, and
+// so is the number of CTA pairs that can be resident), looked up once per device under a lock.
+constexpr int kMaxDevices = 64;
+std::mutex g_launch_mu;
+struct KernelState { bool configured[kMaxDevices]; int pairs[kMaxDevices]; int sms[kMaxDevices]; };
+
+template <typename K>
+cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, int* sms) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_launch_mu);
+    if (!st.configured[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        if (CG == 2) {
-            pairs = max_pairs(kern, SMEM);
-            if (pairs < 1) return cudaErrorInvalidConfiguration;
-        }
-        configured = true;
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        st.sms[dev] = n;
+        st.pairs[dev] = cg == 2 ? max_pairs(kern, smem) : 0;
+        st.configured[dev] = true;
     }
-    const int tiles = ((a.W + TILE_W - 1) / TILE_W) * ((a.H + TILE_H - 1) / TILE_H);
+    *pairs = st.pairs[dev];
+    *sms = st.sms[dev];
+    return cudaSuccess;
+}
+
+template <int BN, bool IB, int OM, int CG, bool PH = false>
+cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
+    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH>;
+    constexpr int SMEM = TileCfg<BN, CG, PH>::SMEM_TOTAL;
+    static KernelState state = {};
+    int pairs = 0, sms = 0;
+    cudaError_t e = kernel_state(kern, SMEM, CG, state, &pairs, &sms);
+    if (e != cudaSuccess) return e;
+    if (CG == 2 && pairs < 1) return cudaErrorInvalidConfiguration;
+    // The phase form tiles the SOURCE grid (its four parities cover the 2x output): the kernel sees a
+    // stride-1 convolution at the source resolution; only its output maps know about the 2x grid.
+    ConvArgs ka = a;
+    if (PH) { ka.H = a.Hs; ka.W = a.Ws; ka.upsample = 0; }
+    const int tiles = ((ka.W + TILE_W - 1) / TILE_W) * ((ka.H + TILE_H - 1) / TILE_H);
     const long long total = (long long)tiles * (padded_cout(a.Cout) / BN) * a.B;
     int grid;
     if (CG == 2) grid = 2 * (int)std::min<long long>((total + 1) / 2, std::min(pairs, kConvMaxCtas / 2));
-    else grid = (int)std::min<long long>(total, std::min(num_sms(), kConvMaxCtas));
-    static const int grid_cap = getenv("VD_CONV_GRID") ? atoi(getenv("VD_CONV_GRID")) : 0;                      // timing studies
-    if (grid_cap > 0) grid = std::max(CG, std::min(grid, grid_cap / CG * CG));
+    else grid = (int)std::min<long long>(total, std::min(sms, kConvMaxCtas));
     // reciprocals for the kernel's tile numbering (see Sched)
-    ConvArgs ka = a;
     {
-        const int tiles_x = (a.W + TILE_W - 1) / TILE_W, nblk = padded_cout(a.Cout) / BN;
+        const int tiles_x = (ka.W + TILE_W - 1) / TILE_W, nblk = padded_cout(a.Cout) / BN;
         const int dmax = std::max(tiles, std::max(tiles_x, nblk));
         if ((unsigned long long)total * (unsigned long long)std::max(dmax, grid + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
         auto recip = [](int d) { return d == 1 ? 0u : (unsigned int)(((1ull << 32) + (unsigned long long)d - 1) / (unsigned long long)d); };
@@ -1210,6 +1309,15 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
                               *(const CUtensorMap*)plan.tmap_y, status);
 }
 
+// can this device co-schedule the CTA pairs of the two-CTA kernels?  (looked up once per device)
+bool pairs_available() {
+    static KernelState state = {};
+    int pairs = 0, sms = 0;
+    auto k = conv_tc_kernel<256, false, 1, 2>;
+    if (kernel_state(k, TileCfg<256, 2>::SMEM_TOTAL, 2, state, &pairs, &sms) != cudaSuccess) { cudaGetLastError(); return false; }
+    return pairs >= 1;
+}
+
 }  // namespace
 
 bool conv_tc_supported(const ConvArgs& a) {
@@ -1217,14 +1325,28 @@ bool conv_tc_supported(const ConvArgs& a) {
     if (!a.bf16_operands) return false;
     if (a.ksize != 1 && a.ksize != 3) return false;
     if (a.x2 && (a.Cin2 % 64 != 0 || a.Cin2 < 64)) return false;
+    if (a.upsample == 2)     // phase-collapsed form: 3x3, 128-channel blocks, plain NHWC store
+        return a.ksize == 3 && a.Cout % 128 == 0 && !a.out_nchw && !a.residual && !a.x2;
     if (a.Cout % 128 == 0) return !a.out_nchw;
     return a.Cout <= 16 && a.out_nchw && !a.residual && !a.x2;      // the frame head: Cout padded to 16
 }
 
-size_t conv_tc_packed_bytes(int Cout, int Cin, int taps) { return (size_t)taps * padded_cout(Cout) * Cin * 2; }
+bool conv_tc_pairs_available() { return pairs_available(); }
+
+size_t conv_tc_packed_bytes(int Cout, int Cin, int taps, bool phase) {
+    return phase ? (size_t)16 * Cout * Cin * 2 : (size_t)taps * padded_cout(Cout) * Cin * 2;
+}
 
 cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int Cout, int Cin, int taps, int cout_total,
-                                  int cout_offset, cudaStream_t s) {
+                                  int cout_offset, bool phase, cudaStream_t s) {
+    if (phase) {
+        if (taps != 9 || cout_offset != 0 || cout_total != Cout || Cout % 128 != 0) return cudaErrorInvalidValue;
+        const int64_t n = (int64_t)16 * Cout * Cin;
+        const int grid = (int)std::min<int64_t>((n + 255) / 256, 148 * 16);
+        if (w_dtype == VD_BF16) pack_weight_phase_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)packed, Cout, Cin);
+        else pack_weight_phase_kernel<float><<<grid, 256, 0, s>>>((const float*)w, (__nv_bfloat16*)packed, Cout, Cin);
+        return cudaGetLastError();
+    }
     const int cpad = padded_cout(cout_total);
     if (cpad != cout_total && cout_offset == 0) {
         cudaError_t e = cudaMemsetAsync(packed, 0, (size_t)taps * cpad * Cin * 2, s);
@@ -1242,22 +1364,45 @@ cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int 
 
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     const int taps = a.ksize * a.ksize;
-    const int bn = pick_bn(a.Cout);
-    // 256-channel blocks run as two-CTA pairs (each CTA loads half of the rows of a weight tile)
-    static const char* pairs_env = getenv("VD_CONV_PAIRS");                 // timing studies: none | up | all
-    const int pairs_mode = !pairs_env ? 1 : (pairs_env[0] == 'n' ? 0 : (pairs_env[0] == 'a' ? 2 : 1));
-    int cg = (bn == 256 && (pairs_mode == 2 || (pairs_mode == 1 && a.upsample))) ? 2 : 1;
-    if (cg == 2) {       // the device must be able to co-schedule pairs of these CTAs; else the one-CTA form
-        static int probe = -1;
-        if (probe < 0) {
-            auto k = conv_tc_kernel<256, false, 1, 2>;
-            probe = (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, TileCfg<256, 2>::SMEM_TOTAL) == cudaSuccess)
-                        ? max_pairs(k, TileCfg<256, 2>::SMEM_TOTAL) : 0;
-            cudaGetLastError();
-        }
-        if (probe < 1) cg = 1;
+    const bool phase = a.upsample == 2;
+    const int bn = phase ? 128 : pick_bn(a.Cout);
+    // 256-channel blocks of the folded upsampling form and the phase form run as two-CTA pairs (each CTA loads
+    // half of the rows of a weight tile); the device must be able to co-schedule such pairs
+    int cg = (phase || (bn == 256 && a.upsample)) ? 2 : 1;
+    if (cg == 2 && !pairs_available()) {
+        if (phase) return cudaErrorInvalidConfiguration;     // the phase form has no one-CTA variant
+        cg = 1;
     }
     plan->cg = cg;
+    plan->phase = phase ? 1 : 0;
+    EncodeTiledFn enc = get_encode_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const bool ob = a.out_dtype == VD_BF16;
+    const cuuint64_t es = ob ? 2 : 4;
+    if (phase) {
+        // weights: 16 * Cout rows in the order pack_weight_phase_kernel writes; one box = a stage of this CTA
+        if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, 16 * a.Cout, 128)) return cudaErrorInvalidValue;
+        // output [B][2 Hs][2 Ws][Cout] seen per row parity a as a 5-D tensor (channel, column parity b, source
+        // column j, source row i, frame): element (c, b, j, i, n) is output pixel (2i + a, 2j + b).  A box is one
+        // epilogue warp's four source rows x 8 source columns of one parity; the store clips the ragged edge.
+        const cuuint64_t W = (cuuint64_t)a.W, C = (cuuint64_t)a.Cout;
+        const cuuint64_t dims[5] = {C, 2, (cuuint64_t)a.Ws, (cuuint64_t)a.Hs, (cuuint64_t)std::max(a.B, 1)};
+        const cuuint64_t strides[4] = {C * es, 2 * C * es, 2 * W * C * es, (cuuint64_t)a.H * W * C * es};
+        const cuuint32_t box[5] = {ob ? 64u : 32u, 1, (cuuint32_t)TILE_W, 4, 1};
+        const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        for (int pa = 0; pa < 2; ++pa) {
+            void* base = (char*)a.y + (size_t)pa * W * C * es;
+            if (enc((CUtensorMap*)(pa ? plan->tmap2 : plan->tmap_y), ob ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                    5, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+        }
+        plan->bn = bn;
+        plan->batch = a.B;
+        plan->y = a.y;
+        plan->valid = 1;
+        return cudaSuccess;
+    }
     if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, taps * padded_cout(a.Cout), bn / cg)) return cudaErrorInvalidValue;
     if (a.x2) {
         if (!encode_weights((CUtensorMap*)plan->tmap2, a.w2, a.Cin2, a.Cout, bn / cg)) return cudaErrorInvalidValue;
@@ -1266,10 +1411,6 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     }
     if (!a.out_nchw) {
         // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one epilogue warp's quarter (4 rows) of a 128-byte-wide slice of a tile
-        EncodeTiledFn enc = get_encode_fn();
-        if (!enc) return cudaErrorNotSupported;
-        const bool ob = a.out_dtype == VD_BF16;
-        const cuuint64_t es = ob ? 2 : 4;
         const cuuint64_t dims[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)std::max(a.B, 1)};
         const cuuint64_t strides[3] = {(cuuint64_t)a.Cout * es, (cuuint64_t)a.W * a.Cout * es, (cuuint64_t)a.H * a.W * a.Cout * es};
         const cuuint32_t box[4] = {ob ? 64u : 32u, (cuuint32_t)TILE_W, 4, 1};      // one epilogue warp's rows
@@ -1288,15 +1429,18 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     return cudaSuccess;
 }
 
-unsigned long long* g_conv_trace = nullptr;   // debug hook, see vd_debug_conv_trace
-
-cudaError_t launch_conv_tc(const ConvArgs& a_in, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
+cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
     if (!plan.valid) return cudaErrorInvalidValue;
-    ConvArgs a = a_in;
-    a.trace = g_conv_trace;
     if (!a.out_nchw && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
+    if ((a.upsample == 2) != (plan.phase != 0)) return cudaErrorInvalidValue;
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
+    if (plan.phase) {
+        if (ib && ob) return launch_one<128, true, 1, 2, true>(a, plan, status, s);
+        if (ib && !ob) return launch_one<128, true, 0, 2, true>(a, plan, status, s);
+        if (!ib && ob) return launch_one<128, false, 1, 2, true>(a, plan, status, s);
+        return launch_one<128, false, 0, 2, true>(a, plan, status, s);
+    }
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
     }

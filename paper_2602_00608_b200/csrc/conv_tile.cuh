@@ -1,5 +1,5 @@
 // Pieces shared by the one-CTA and the two-CTA tensor-core convolution kernels: tile geometry,
-// the operand loader of the prologue, and the debug timeline recorder.
+// and the operand loader of the prologue.
 #pragma once
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -22,11 +22,10 @@ static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the ha
 // MMA-issuing thread no priority: measured, fifteen warps of dense arithmetic stretch its
 // wait / 4 x MMA / commit sequence from 513 to about 1800 cycles, while the same warps kept off its
 // sub-partition cost nothing.  So sub-partition 0 carries only the MMA warp, the TMA warp and one
-// epilogue warp (warp 8 is the optional second MMA warp of two-tile items (off by default), warp 12 prefetches inputs into L2; warp 20 idles until the end), and the fifteen producer warps are the
+// epilogue warp (warp 12 prefetches inputs into L2; warps 8 and 20 idle until the end), and the fifteen producer warps are the
 // warps with warp % 4 != 0 outside the epilogue: five per remaining sub-partition.
 constexpr int MMA_WARP = 0;
 constexpr int PREFETCH_WARP = 12;                                   // asks L2 for the next item's input rows
-constexpr int MMA_WARP2 = 8;                                        // second issuing thread where an item is two tiles
 constexpr int TMA_WARP = 4;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
 constexpr int NUM_THREADS = 24 * 32;
@@ -77,37 +76,6 @@ __device__ __forceinline__ void unpack_raw(bool is_bf16, const Raw8& r, float v[
 }
 
 struct Tile { int tx0, ty0, n0, b; };
-
-// Debug timeline (builds with -DVD_CONV_TRACE only): role r of this CTA appends (code << 48 | clock)
-// records when a trace buffer is given.
-struct Tracer {
-    unsigned long long* p;
-    int n;
-#ifdef VD_CONV_TRACE
-    // VD_CONV_TRACE is a mask of the roles that record (bit = role number), so that one role can
-    // be observed while the others run the production code
-    __device__ __forceinline__ void init(unsigned long long* base, int role) {
-        p = (base && ((VD_CONV_TRACE >> role) & 1)) ? base + ((size_t)blockIdx.x * 4 + role) * kConvTraceEvents : nullptr;
-        n = 0;
-    }
-    __device__ __forceinline__ void mark(unsigned code) {
-        if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clock64() & 0xFFFFFFFFFFFFull);
-    }
-    __device__ __forceinline__ void mark_fine(unsigned code) {       // per-tap marks of the MMA thread: bit 4 of the mask
-        if ((VD_CONV_TRACE >> 4) & 1) mark(code);
-    }
-    __device__ __forceinline__ void mark_at(unsigned code, long long clk) {
-        if (p && n < kConvTraceEvents) p[n++] = ((unsigned long long)code << 48) | ((unsigned long long)clk & 0xFFFFFFFFFFFFull);
-    }
-    static __device__ __forceinline__ long long now() { return clock64(); }
-#else   // production builds carry no tracing code at all (the MMA-issuing thread is latency critical)
-    __device__ __forceinline__ void init(unsigned long long*, int) {}
-    __device__ __forceinline__ void mark(unsigned) {}
-    __device__ __forceinline__ void mark_fine(unsigned) {}
-    __device__ __forceinline__ void mark_at(unsigned, long long) {}
-    static __device__ __forceinline__ long long now() { return 0; }
-#endif
-};
 
 }  // namespace convtile
 }  // namespace vd

@@ -557,7 +557,8 @@ cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cud
 // asynchronous memset at the start of every call.
 namespace {
 constexpr int kStaticGnMaxBatchTimesGroups = 64;     // e.g. 2 frames x 32 groups, or 8 x 8
-static __device__ __align__(256) float g_gn_static_partial[kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2 + 64];   // 148 KiB of chunk records + 64 arrival counters
+constexpr int kStaticGnCounters = 64;                // arrival counters behind the records (batch <= 64 follows from the limit)
+static __device__ __align__(256) float g_gn_static_partial[kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2 + kStaticGnCounters];   // 148 KiB of chunk records + 64 arrival counters
 
 std::mutex g_static_mu;
 constexpr int kMaxDevices = 64;
@@ -594,6 +595,10 @@ extern "C" VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, 
         set_last_error("vd_op_gn_stats_static: bad GroupNorm sizes (groups must hold a multiple of 4 channels)");
         return VD_ERR_INVALID_ARG;
     }
+    if ((long long)h * w > 0x7fffffffLL || (long long)batch * h * w * c > (1LL << 40)) {
+        set_last_error("vd_op_gn_stats_static: tensor too large (h*w must fit 31 bits, batch*h*w*c 40 bits)");
+        return VD_ERR_INVALID_ARG;
+    }
     if ((long long)batch * groups > kStaticGnMaxBatchTimesGroups) {
         set_last_error("vd_op_gn_stats_static: batch*groups exceeds 64, the capacity of the built-in scratch array; "
                        "use vd_op_gn_stats with a scratch buffer instead");
@@ -605,7 +610,7 @@ extern "C" VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, 
     if (e == cudaSuccess) {
         // the arrival counters live behind the records; they must be zero when the kernel starts
         unsigned int* counters = (unsigned int*)(partial + (size_t)kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2);
-        e = cudaMemsetAsync(counters, 0, 64 * sizeof(unsigned int), (cudaStream_t)cuda_stream);
+        e = cudaMemsetAsync(counters, 0, kStaticGnCounters * sizeof(unsigned int), (cudaStream_t)cuda_stream);
         GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial, counters};
         if (e == cudaSuccess) e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
     }

@@ -31,6 +31,7 @@ struct WeightJob {           // repack work done once in vd_create
     std::string name;        // source tensor
     int kind;                // 0 conv weight (packed), 1 vector -> fp32
     bool tc;
+    bool phase;              // tensor-core weights of the phase-collapsed upsampling form
     int Cout, Cin, taps;
     int cout_total, cout_offset;
     size_t dst_off;
@@ -74,24 +75,24 @@ class Planner {
     struct ConvW { size_t w_off, b_off; bool tc; };
 
     // registers the repack of a conv weight (possibly a stack of several source tensors along Cout)
-    ConvW conv_weight(const std::vector<std::string>& names, int Cout_each, int Cin, int taps, bool tc) {
+    ConvW conv_weight(const std::vector<std::string>& names, int Cout_each, int Cin, int taps, bool tc, bool phase = false) {
         const int Cout = Cout_each * (int)names.size();
         ConvW r;
         r.tc = tc;
-        const size_t wbytes = tc ? conv_tc_packed_bytes(Cout, Cin, taps) : (size_t)taps * Cin * Cout * 4;
+        const size_t wbytes = tc ? conv_tc_packed_bytes(Cout, Cin, taps, phase) : (size_t)taps * Cin * Cout * 4;
         r.w_off = alloc(wbytes);
         r.b_off = alloc((size_t)Cout * 4);
         for (size_t i = 0; i < names.size(); ++i) {
-            h_->jobs.push_back({names[i] + ".weight", 0, tc, Cout_each, Cin, taps, Cout, (int)i * Cout_each, r.w_off});
-            h_->jobs.push_back({names[i] + ".bias", 1, false, Cout_each, 0, 0, 0, 0, r.b_off + (size_t)i * Cout_each * 4});
+            h_->jobs.push_back({names[i] + ".weight", 0, tc, phase, Cout_each, Cin, taps, Cout, (int)i * Cout_each, r.w_off});
+            h_->jobs.push_back({names[i] + ".bias", 1, false, false, Cout_each, 0, 0, 0, 0, r.b_off + (size_t)i * Cout_each * 4});
         }
         return r;
     }
     void norm_weight(const std::string& name, int C, size_t& g_off, size_t& b_off) {
         g_off = alloc((size_t)C * 4);
         b_off = alloc((size_t)C * 4);
-        h_->jobs.push_back({name + ".weight", 1, false, C, 0, 0, 0, 0, g_off});
-        h_->jobs.push_back({name + ".bias", 1, false, C, 0, 0, 0, 0, b_off});
+        h_->jobs.push_back({name + ".weight", 1, false, false, C, 0, 0, 0, 0, g_off});
+        h_->jobs.push_back({name + ".bias", 1, false, false, C, 0, 0, 0, 0, b_off});
     }
 
     void add_gn(const std::string& name, size_t x_off, int dtype, int H, int W, int C, const std::string& wname) {
@@ -129,13 +130,22 @@ class Planner {
         a.residual = residual_off >= 0 ? ptr<float>((size_t)residual_off) : nullptr;
         a.y = y_is_frames ? nullptr : ptr<void>(y_off);
         a.B = 0; a.Hs = Hs; a.Ws = Ws; a.H = H; a.W = W;
-        a.Cin = Cin; a.Cout = Cout; a.ksize = ksize; a.upsample = upsample; a.silu = silu;
+        a.Cin = Cin; a.Cout = Cout; a.ksize = ksize; a.upsample = upsample ? 1 : 0; a.silu = silu;
         a.in_dtype = in_dtype; a.out_dtype = out_dtype; a.out_nchw = out_nchw; a.bf16_operands = bf16();
         if (!shortcut_name.empty()) { a.x2 = ptr<void>(x2_off); a.Cin2 = Cin2; }
+        const bool tc_on = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT);
         ConvArgs probe = a;
         probe.B = 1;
-        const bool tc = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && conv_tc_supported(probe);
-        ConvW cw = conv_weight(wnames, Cout_each, Cin, ksize * ksize, tc);
+        // an upsampling 3x3 runs in the phase-collapsed form (4/9 of the products) where the tensor-core kernel has it
+        bool phase = false;
+        if (tc_on && upsample && !(cfg_.flags & VD_FLAG_UPSAMPLE_9TAP)) {
+            probe.upsample = 2;
+            phase = conv_tc_supported(probe);
+            if (!phase) probe.upsample = 1;
+        }
+        if (phase) a.upsample = 2;
+        const bool tc = tc_on && conv_tc_supported(probe);
+        ConvW cw = conv_weight(wnames, Cout_each, Cin, ksize * ksize, tc, phase);
         a.w = ptr<void>(cw.w_off);
         a.bias = ptr<float>(cw.b_off);
         if (!shortcut_name.empty()) {          // only requested when the tensor-core kernel takes this layer
@@ -153,6 +163,7 @@ class Planner {
                                  (residual_off >= 0 ? P * Cout * 4.0 : 0.0);
         s.info.weight_bytes = (double)ksize * ksize * Cin * Cout * elt(cfg_.dtype);
         s.info.has_residual = residual_off >= 0;
+        s.info.phase_collapsed = phase ? 1 : 0;
         if (!shortcut_name.empty()) {
             s.info.c_in2 = Cin2;
             s.info.flops_per_frame += 2.0 * Cin2 * (double)Cout * P;
@@ -360,7 +371,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~VD_FLAG_FORCE_SIMT) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -412,10 +423,7 @@ cudaError_t launch_step(const vd_handle_s* h, const Step& st, int B, const void*
 
 namespace vd {
 static thread_local bool t_pdl_active = false;
-bool pdl_enabled() {
-    static const bool off = getenv("VD_NO_PDL") != nullptr;
-    return t_pdl_active && !off;
-}
+bool pdl_enabled() { return t_pdl_active; }
 PdlScope::PdlScope(bool on) : prev(t_pdl_active) { t_pdl_active = on; }
 PdlScope::~PdlScope() { t_pdl_active = prev; }
 }  // namespace vd
@@ -464,7 +472,6 @@ vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, floa
 }  // namespace
 
 namespace vd {
-extern unsigned long long* g_conv_trace;
 void set_last_error(const char* msg) { g_last_error = msg ? msg : ""; }
 }  // namespace vd
 
@@ -531,7 +538,7 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
         if (j.kind == 1) {
             e = launch_to_f32(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, s);
         } else if (j.tc) {
-            e = launch_pack_weight_tc(t->dptr, t->dtype, h->ws + j.dst_off, j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, s);
+            e = launch_pack_weight_tc(t->dptr, t->dtype, h->ws + j.dst_off, j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, j.phase, s);
         } else {
             e = launch_pack_weight_simt(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, s);
         }
@@ -542,6 +549,11 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
             ConvArgs pa = st.conv;
             pa.B = cfg->max_batch;
             e = conv_tc_prepare(pa, &st.tc);
+            if (e == cudaErrorInvalidConfiguration && pa.upsample == 2) {
+                delete h;
+                return fail(nullptr, VD_ERR_UNSUPPORTED, "this device cannot co-schedule the CTA pairs of the phase-collapsed "
+                                                         "upsampling convolution; set VD_FLAG_UPSAMPLE_9TAP");
+            }
             if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "weight tensor map"); }
         }
     }
@@ -589,10 +601,18 @@ vd_status vd_get_status(vd_handle h) {
     if (e != cudaSuccess) return cuda_fail(h, e, "status read");
     if (word[0] != 0) {
         char msg[160];
-        snprintf(msg, sizeof(msg), "a kernel gave up on a bounded wait (code 0x%x, block %u, detail 0x%x)", word[0], word[1], word[2]);
+        const char* who = word[0] == kStatusConvTimeout ? "convolution" : word[0] == kStatusAttnTimeout ? "attention"
+                          : word[0] == kStatusWaitProbe ? "wait probe" : "unknown";
+        snprintf(msg, sizeof(msg), "a %s kernel gave up on a bounded wait (code 0x%x, block %u, detail 0x%x)", who, word[0], word[1], word[2]);
         return fail(h, VD_ERR_DEVICE_TIMEOUT, msg);
     }
     return VD_OK;
+}
+
+vd_status vd_clear_status(vd_handle h, void* cuda_stream) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    cudaError_t e = cudaMemsetAsync(h->ws + h->status_off, 0, 256, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(h, e, "status clear");
 }
 
 const char* vd_last_error(vd_handle h) { return h ? h->err.c_str() : g_last_error.c_str(); }
@@ -622,11 +642,18 @@ vd_status vd_profile(vd_handle h, const void* latents, void* frames, int32_t bat
     return decode_impl(h, latents, nullptr, 0.f, nullptr, nullptr, frames, batch, cuda_stream, ms, n_steps);
 }
 
-vd_status vd_debug_conv_trace(void* device_buffer, size_t bytes) {
-    if (device_buffer && bytes < (size_t)kConvMaxCtas * 4 * kConvTraceEvents * sizeof(unsigned long long))
-        return fail(nullptr, VD_ERR_INVALID_ARG, "trace buffer too small");
-    vd::g_conv_trace = (unsigned long long*)device_buffer;
+vd_status vd_debug_status_offset(vd_handle h, int64_t* offset) {
+    if (!h || !offset) return fail(h, VD_ERR_INVALID_ARG, "NULL argument");
+    *offset = (int64_t)h->status_off;
     return VD_OK;
+}
+
+vd_status vd_debug_wait_probe(vd_handle h, int64_t limit_cycles, void* cuda_stream) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (limit_cycles < 1000 || limit_cycles > 2000000000LL)
+        return fail(h, VD_ERR_INVALID_ARG, "limit_cycles must be in [1e3, 2e9]");
+    cudaError_t e = launch_wait_probe((unsigned int*)(h->ws + h->status_off), (long long)limit_cycles, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(h, e, "vd_debug_wait_probe");
 }
 
 vd_status vd_debug_stop_after(vd_handle h, int32_t index) {
@@ -644,6 +671,7 @@ static vd_status check_conv_desc(const vd_conv_desc* d) {
     if ((d->in_dtype != VD_F32 && d->in_dtype != VD_BF16) || (d->out_dtype != VD_F32 && d->out_dtype != VD_BF16))
         return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
     if (d->impl < VD_IMPL_AUTO || d->impl > VD_IMPL_TC) return fail(nullptr, VD_ERR_INVALID_ARG, "bad impl");
+    if (d->upsample < 0 || d->upsample > 2) return fail(nullptr, VD_ERR_INVALID_ARG, "upsample must be 0, 1 or 2");
     return VD_OK;
 }
 
@@ -652,7 +680,7 @@ static ConvArgs conv_args_from_desc(const vd_conv_desc* d) {
     a.B = d->batch; a.Hs = d->in_h; a.Ws = d->in_w;
     a.H = d->upsample ? 2 * d->in_h : d->in_h;
     a.W = d->upsample ? 2 * d->in_w : d->in_w;
-    a.Cin = d->c_in; a.Cout = d->c_out; a.ksize = d->ksize; a.upsample = d->upsample ? 1 : 0; a.silu = d->silu ? 1 : 0;
+    a.Cin = d->c_in; a.Cout = d->c_out; a.ksize = d->ksize; a.upsample = d->upsample; a.silu = d->silu ? 1 : 0;
     a.in_dtype = d->in_dtype; a.out_dtype = d->out_dtype; a.out_nchw = d->out_nchw ? 1 : 0;
     a.bf16_operands = d->bf16_operands ? 1 : 0;
     return a;
@@ -664,6 +692,7 @@ static vd_status resolve_impl(const vd_conv_desc* d, const ConvArgs& a, bool* tc
     const bool can = a.bf16_operands && conv_tc_supported(probe);
     if (d->impl == VD_IMPL_TC && !can) return fail(nullptr, VD_ERR_UNSUPPORTED, "the tensor-core convolution does not support this shape");
     *tc = d->impl == VD_IMPL_TC || (d->impl == VD_IMPL_AUTO && can);
+    if (!*tc && a.upsample == 2) return fail(nullptr, VD_ERR_UNSUPPORTED, "the phase-collapsed upsampling form exists in the tensor-core kernel only");
     return VD_OK;
 }
 
@@ -675,7 +704,7 @@ vd_status vd_conv_packed_weight_bytes(const vd_conv_desc* d, size_t* bytes) {
     st = resolve_impl(d, conv_args_from_desc(d), &tc);
     if (st != VD_OK) return st;
     const int taps = d->ksize * d->ksize;
-    *bytes = tc ? conv_tc_packed_bytes(d->c_out, d->c_in, taps) : (size_t)taps * d->c_in * d->c_out * 4;
+    *bytes = tc ? conv_tc_packed_bytes(d->c_out, d->c_in, taps, d->upsample == 2) : (size_t)taps * d->c_in * d->c_out * 4;
     return VD_OK;
 }
 
@@ -688,7 +717,7 @@ vd_status vd_conv_pack_weight(const vd_conv_desc* d, const void* w_oihw, int32_t
     st = resolve_impl(d, conv_args_from_desc(d), &tc);
     if (st != VD_OK) return st;
     const int taps = d->ksize * d->ksize;
-    cudaError_t e = tc ? launch_pack_weight_tc(w_oihw, w_dtype, packed, d->c_out, d->c_in, taps, d->c_out, 0, (cudaStream_t)cuda_stream)
+    cudaError_t e = tc ? launch_pack_weight_tc(w_oihw, w_dtype, packed, d->c_out, d->c_in, taps, d->c_out, 0, d->upsample == 2, (cudaStream_t)cuda_stream)
                        : launch_pack_weight_simt(w_oihw, w_dtype, (float*)packed, d->c_out, d->c_in, taps, d->c_out, 0, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_conv_pack_weight");
 }
@@ -736,6 +765,8 @@ vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h,
     if (dtype != VD_F32 && dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
     if (batch < 0 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups != 0 || (c / groups) % 4 != 0 || c > 1024)
         return fail(nullptr, VD_ERR_INVALID_ARG, "bad GroupNorm sizes (groups must hold a multiple of 4 channels)");
+    if ((long long)h * w > 0x7fffffffLL || (long long)batch * h * w * c > (1LL << 40))
+        return fail(nullptr, VD_ERR_INVALID_ARG, "tensor too large (h*w must fit 31 bits, batch*h*w*c 40 bits)");
     if (batch == 0) return VD_OK;
     unsigned int* counters = (unsigned int*)((char*)scratch + gn_partial_bytes(batch, groups));
     GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch, counters};

@@ -6,7 +6,7 @@
 
 #include <utility>
 
-#include "vd.h"
+#include "vd_ops.h"
 
 namespace vd {
 
@@ -21,20 +21,21 @@ struct ConvArgs {
     void* y;                // out_dtype, NHWC [B,H,W,Cout] or NCHW [B,Cout,H,W]
     int B, Hs, Ws;          // source resolution
     int H, W;               // output resolution (= source, or 2x source with upsample)
-    int Cin, Cout, ksize, upsample, silu;
+    int Cin, Cout, ksize;
+    int upsample;           // 0 none; 1 nearest-2x folded into the addressing (9 taps on the 2x grid); 2 phase-collapsed
+                            // (four 2x2 convolutions of the source with pre-summed weights; tensor-core kernel only)
+    int silu;
     int in_dtype, out_dtype, out_nchw, bf16_operands;
     // optional fused 1x1 shortcut (tensor-core kernel only): y += W2 * x2 + bias2
     const void* x2;         // fp32 NHWC [B,H,W,Cin2] at the output resolution, or null
     const void* w2;         // packed bf16 [Cout][Cin2]
     const float* bias2;     // [Cout] or null
     int Cin2;
-    unsigned long long* trace;  // debug: per-CTA role timelines (null in production)
     // tensor-core kernel: ceil(2^32 / d) for the divisors of its tile numbering (tiles per image, channel
     // blocks, tiles per row), filled in by its launcher; 0 stands for d = 1
     unsigned int div_tiles, div_nblk, div_tx;
 };
-constexpr int kConvTraceEvents = 2048;    // per (CTA, role)
-constexpr int kConvMaxCtas = 160;         // upper bound on the persistent grid (sizes the debug trace)
+constexpr int kConvMaxCtas = 160;         // upper bound on the persistent grid
 
 struct GnArgs {
     const void* x;          // NHWC [B,H,W,C]
@@ -71,6 +72,10 @@ struct IngestArgs {
     int dtype, B, C, h, w;
 };
 
+// codes the kernels latch in the status word when a bounded wait runs out
+constexpr unsigned int kStatusConvTimeout = 0xC0DE0001u, kStatusAttnTimeout = 0xC0DE0002u, kStatusWaitProbe = 0xC0DE0003u;
+cudaError_t launch_wait_probe(unsigned int* status_word, long long limit_cycles, cudaStream_t s);   // wait_probe.cu
+
 // records `msg` as the text vd_last_error(NULL) returns (defined in vd_api.cu)
 void set_last_error(const char* msg);
 
@@ -88,10 +93,12 @@ cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cud
 
 // ---- tcgen05 kernels (conv_tc.cu, attn_tc.cu)
 bool conv_tc_supported(const ConvArgs& a);
-size_t conv_tc_packed_bytes(int Cout, int Cin, int taps);
-// OIHW weight (bf16) -> bf16 [tap][Cout_pad][Cin] (K-major rows for the B operand)
+bool conv_tc_pairs_available();          // can the current device co-schedule the kernels' CTA pairs?
+size_t conv_tc_packed_bytes(int Cout, int Cin, int taps, bool phase);
+// OIHW weight (bf16) -> bf16 [tap][Cout_pad][Cin] (K-major rows for the B operand); phase: the sixteen
+// pre-summed 2x2 taps of the phase-collapsed upsampling convolution, in the order its kernel streams them
 cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int Cout, int Cin, int taps,
-                                  int cout_total, int cout_offset, cudaStream_t s);
+                                  int cout_total, int cout_offset, bool phase, cudaStream_t s);
 // Launch-invariant state of one tensor-core convolution: the TMA descriptor of its packed weights.
 struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
@@ -101,6 +108,7 @@ struct alignas(64) ConvTcPlan {
     int batch;                  // frames covered by tmap_y
     int bn;
     int cg;                     // CTAs per MMA: 2 = two-CTA pairs (weight maps built with half-height boxes)
+    int phase;                  // 1: phase-collapsed upsampling form (tmap_y / tmap2 are the output maps of row parity 0 / 1)
     int valid;
 };
 cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w must be the final packed-weight address
@@ -120,7 +128,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStr
 // written, before the wait.
 // Dependent launches are used only inside a PdlScope (the decode loop): the single-operator entry
 // points launch plainly, since their inputs may come from work this library knows nothing about.
-bool pdl_enabled();     // inside a PdlScope, and the environment variable VD_NO_PDL is not set
+bool pdl_enabled();     // inside a PdlScope
 struct PdlScope {
     explicit PdlScope(bool on);
     ~PdlScope();

@@ -1,13 +1,17 @@
-"""Writes tests/golden/frames_cfg{3,4,5}.npz: oracle frames of the full-size workloads, sampled.
+"""Writes the oracle frames of the full-size workloads that the GPU parity tests compare with.
 
-Calls only the oracle (`oracle/`) and the seeded input generators.  For every frame of the
-workload the whole decoder is run by the oracle; kept are all three channels at a fixed set of
-pixel positions (image corners, points along the four borders, and seeded random positions),
-plus each frame's mean, standard deviation and L2 norm.  Run from the repository root:
+Calls only the oracle (`oracle/`) and the seeded input generators.
 
-    python tests/golden/make_golden.py 3 4 5
+    python tests/golden/make_golden.py 3 4 5          # frames_cfg{3,4,5}.npz
+    python tests/golden/make_golden.py --full 3 4 5   # frame_cfg{3,4,5}_full.npz
 
-About 80 s of an 8-core host per 720x480 frame.
+Without --full: for every frame of the workload the whole decoder is run by the oracle; kept are
+all three channels at a fixed set of pixel positions (image corners, points along the four
+borders, and seeded random positions), plus each frame's mean, standard deviation and L2 norm.
+With --full: the LAST frame of the workload is kept whole (every pixel, fp32), so that the
+max-abs bar can be checked over the complete frame.
+
+About 90 s of an 8-core host per 720x480 frame, 280 s per 1280x720 one.
 """
 import os
 import sys
@@ -56,5 +60,22 @@ def main(indices):
         print("wrote", out, os.path.getsize(out), "bytes", flush=True)
 
 
+def main_full(indices):
+    for idx in indices:
+        wl = synth.WORKLOADS[idx]
+        wts = synth.workload_weights(wl)
+        z = synth.workload_latents(wl)
+        b = wl.batch - 1
+        t0 = time.time()
+        y = ref.decode(wl.arch, wts, z[b:b + 1], wl.groups, wl.eps)[0]
+        print(f"cfg {idx} frame {b}: {time.time() - t0:.1f} s", flush=True)
+        out = os.path.join(os.path.dirname(os.path.abspath(__file__)), f"frame_cfg{idx}_full.npz")
+        np.savez_compressed(out, frame=y.astype(np.float32), index=np.int32(b))
+        print("wrote", out, os.path.getsize(out), "bytes", flush=True)
+
+
 if __name__ == "__main__":
-    main([int(a) for a in sys.argv[1:]] or [3, 4, 5])
+    argv = sys.argv[1:]
+    full = "--full" in argv
+    idxs = [int(a) for a in argv if a != "--full"] or [3, 4, 5]
+    (main_full if full else main)(idxs)

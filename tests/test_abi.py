@@ -19,7 +19,7 @@ def vd():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "vd.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", f)).read() for f in sorted(os.listdir(os.path.join(ROOT, "include"))))
     return sorted(set(re.findall(r"VD_API\s+[\w\s\*]+?\b(vd_\w+)\s*\(", text)))
 
 

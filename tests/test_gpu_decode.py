@@ -114,6 +114,40 @@ def test_full_size_configs_against_sampled_oracle_frames(env, idx):
     dec.check_status()
 
 
+# measured on one B200 (whole frame, every pixel): see the parity table of the design notes
+@pytest.mark.parametrize("idx", [3, 4, 5])
+def test_full_size_configs_whole_frame_against_the_oracle(env, idx):
+    """The last frame of each full-size workload, complete: every output pixel against the oracle
+    frame that tests/golden/make_golden.py --full stored (oracle only), at the bar of the bf16
+    path; and the tensor-core path against the FFMA path of the same library on every pixel of
+    every frame (the FFMA path is itself checked against the oracle)."""
+    torch, ref, vd, synth = env
+    path = os.path.join(GOLDEN, f"frame_cfg{idx}_full.npz")
+    gold = np.load(path)
+    wl = synth.WORKLOADS[idx]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z)
+    b = int(gold["index"])
+    assert b == wl.batch - 1
+    g = got[b].float().cpu().numpy()
+    want = gold["frame"]
+    assert g.shape == want.shape == (3, wl.out_h, wl.out_w)
+    r, m = rel_l2(g, want), max_abs(g, want)
+    print(f"whole-frame parity {wl.name} frame {b}: rel-L2 {r:.3e} max-abs {m:.3e}")
+    assert r <= BF16_REL_L2 and m <= BF16_MAX_ABS, (r, m)
+    dec.close()
+    del dec
+    torch.cuda.empty_cache()
+    # every pixel of every frame, tcgen05 kernels against the FFMA kernels (same rounding points)
+    zs = z[-2:] if wl.batch > 2 else z                      # the FFMA path is slow: two frames are enough
+    dec2, got2, _ = _decode(env, wl, zs, flags=vd.VD_FLAG_FORCE_SIMT)
+    a = got[-zs.shape[0]:].float()
+    d = (a - got2.float())
+    r2 = float(d.norm() / got2.float().norm())
+    print(f"tcgen05 vs FFMA {wl.name}: rel-L2 {r2:.3e} max-abs {float(d.abs().max()):.3e}")
+    assert r2 <= 6e-3 and float(d.abs().max()) <= BF16_MAX_ABS
+
+
 def test_host_buffer_decode_and_extrapolation(env):
     torch, ref, vd, synth = env
     wl = synth.WORKLOADS[2]

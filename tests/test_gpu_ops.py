@@ -227,6 +227,70 @@ TC_CASES = [
 ]
 
 
+# Phase-collapsed upsampling convolution (upsample=2): per output parity a 2x2 convolution of the source with
+# pre-summed weights.  Ragged source tiles, an odd number of tiles per channel block (the peer CTA of the
+# last pair has none), several channel blocks and frames, 1..8 input chunks, every dtype combination.
+PHASE_CASES = [
+    dict(B=1, H=9, W=13, Cin=128, Cout=256, k=3, upsample=2, prologue=False, silu=False, residual=False, in_bf16=False, out_bf16=False),
+    dict(B=1, H=16, W=24, Cin=64, Cout=128, k=3, upsample=2, prologue=False, silu=False, residual=False, in_bf16=True, out_bf16=False),
+    dict(B=2, H=12, W=11, Cin=128, Cout=512, k=3, upsample=2, prologue=True, silu=True, residual=False, in_bf16=False, out_bf16=True),
+    dict(B=3, H=20, W=30, Cin=512, Cout=128, k=3, upsample=2, prologue=False, silu=False, residual=False, in_bf16=False, out_bf16=False),
+    dict(B=2, H=33, W=17, Cin=256, Cout=256, k=3, upsample=2, prologue=True, silu=False, residual=False, in_bf16=True, out_bf16=True),
+    dict(B=1, H=1, W=1, Cin=64, Cout=128, k=3, upsample=2, prologue=False, silu=False, residual=False, in_bf16=False, out_bf16=False),
+]
+
+
+@pytest.mark.parametrize("case", PHASE_CASES)
+def test_conv_tc_phase_collapsed_upsample_matches_oracle(env, case):
+    _, _, vd, _ = env
+    got, want = _conv_case(env, seed=47, impl=vd.VD_IMPL_TC, bf16_ops=True, **case)
+    assert got.shape == want.shape
+    # as test_conv_tc_matches_oracle, plus one bf16 rounding of every pre-summed weight (another
+    # 2^-9 relative per product, independent of the operand's): sqrt(2) x the one-rounding error
+    tol = 4.5e-3 if case["out_bf16"] else 3e-3
+    assert rel_l2(got, want) <= tol
+    # against the 9-tap folded form of the same kernel family: same operands, weights summed after
+    # instead of before the rounding
+    got9, _ = _conv_case(env, seed=47, impl=vd.VD_IMPL_TC, bf16_ops=True, **dict(case, upsample=1))
+    assert rel_l2(got, got9) <= (4.5e-3 if case["out_bf16"] else 2e-3)
+
+
+@pytest.mark.parametrize("ky,kx", [(ky, kx) for ky in range(3) for kx in range(3)])
+def test_conv_tc_phase_collapsed_single_taps_are_exact(env, ky, kx):
+    """A single 3x3 tap with identity channels: every pre-summed weight is 0 or 1, so the output is
+    the shifted, upsampled bf16 operand bit for bit.  Pins the tap sets of the four parities, the
+    parity of the output coordinates and the zero ring, tap by tap."""
+    torch, ref, vd, synth = env
+    B, H, W, C = 2, 19, 10, 64
+    x = synth.round_to_bf16(_rng(7).standard_normal((B, C, H, W)).astype(np.float32))
+    w = np.zeros((128, C, 3, 3), np.float32)
+    w[np.arange(C), np.arange(C), ky, kx] = 1.0
+    y = vd.op_conv2d(util.nchw_to_dev_nhwc(x, torch.bfloat16), torch.from_numpy(w).cuda().bfloat16(),
+                     upsample=2, out_dtype=vd.VD_F32, bf16_operands=True, impl=vd.VD_IMPL_TC)
+    torch.cuda.synchronize()
+    got = util.dev_nhwc_to_nchw(y)
+    want = ref.conv2d(ref.upsample2x(x), w)
+    assert got.shape == want.shape == (B, 128, 2 * H, 2 * W)
+    assert np.array_equal(got, want)
+
+
+def test_conv_tc_phase_collapsed_all_ones_counts_taps(env):
+    """All-ones input and weights: every output is (number of in-image taps) x Cin: 9 Cin inside,
+    6 Cin on the edges, 4 Cin in the corners of the UPSAMPLED image (sums of small integers are
+    exact in bf16 weights and fp32 accumulation)."""
+    torch, ref, vd, synth = env
+    H, W, C = 5, 7, 64
+    x = np.ones((1, C, H, W), np.float32)
+    w = np.ones((128, C, 3, 3), np.float32)
+    y = vd.op_conv2d(util.nchw_to_dev_nhwc(x, torch.bfloat16), torch.from_numpy(w).cuda().bfloat16(),
+                     upsample=2, out_dtype=vd.VD_F32, bf16_operands=True, impl=vd.VD_IMPL_TC)
+    torch.cuda.synchronize()
+    got = util.dev_nhwc_to_nchw(y)[0, 0]
+    cnt_y = np.full(2 * H, 3.0); cnt_y[[0, -1]] = 2.0
+    cnt_x = np.full(2 * W, 3.0); cnt_x[[0, -1]] = 2.0
+    assert np.array_equal(got, np.outer(cnt_y, cnt_x) * C)
+
+
 @pytest.mark.parametrize("case", TC_CASES)
 def test_conv_tc_matches_oracle(env, case):
     _, _, vd, _ = env

@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
 
 def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row():
     import torch
+    from oracle import ref
     from paper_2602_00608_b200 import binding as vd
 
     gen = np.random.Generator(np.random.Philox(key=99))
@@ -24,12 +25,19 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice_in_a_row():
         gamma = torch.from_numpy(gen.uniform(0.9, 1.1, c).astype(np.float32)).cuda()
         beta = torch.from_numpy(gen.uniform(-0.1, 0.1, c).astype(np.float32)).cuda()
         want_scale, want_shift = vd.op_gn_stats(x, gamma, beta, g, 1e-6)
+        # and against the oracle's two-pass GroupNorm, so that the test stands on its own
+        x_nchw = x.float().permute(0, 3, 1, 2).contiguous().cpu().numpy()
+        _, mean, rstd = ref.groupnorm(x_nchw, gamma.cpu().numpy(), beta.cpu().numpy(), g, 1e-6, return_stats=True)
+        ref_scale = gamma.cpu().numpy()[None, :] * np.repeat(rstd, c // g, axis=1)
+        ref_shift = beta.cpu().numpy()[None, :] - np.repeat(mean, c // g, axis=1) * ref_scale
         for _ in range(2):                                   # second call sees the first call's leftovers
             scale, shift = vd.op_gn_stats_static(x, gamma, beta, g, 1e-6)
             torch.cuda.synchronize()
             # same kernels, same summation order: the tolerance of the statistics tests is far from reached
             np.testing.assert_allclose(scale.cpu().numpy(), want_scale.cpu().numpy(), rtol=2e-5)
             np.testing.assert_allclose(shift.cpu().numpy(), want_shift.cpu().numpy(), rtol=2e-5, atol=2e-5)
+            np.testing.assert_allclose(scale.cpu().numpy(), ref_scale, rtol=2e-5)
+            np.testing.assert_allclose(shift.cpu().numpy(), ref_shift, rtol=2e-5, atol=2e-5)
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
