@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--residual", action="store_true")
     ap.add_argument("--prologue", action="store_true")
     ap.add_argument("--upsample", action="store_true")
+    ap.add_argument("--phase", action="store_true", help="with --upsample: the phase-collapsed form (upsample=2)")
     ap.add_argument("--nchw", action="store_true")
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
@@ -48,7 +49,7 @@ def main():
     shift = torch.zeros((a.batch, a.cin), device="cuda") if a.prologue else None
     od = vd.VD_F32 if a.out_f32 else vd.VD_BF16
 
-    d = vd.conv_desc(a.batch, a.h, a.w, a.cin, a.cout, a.k, a.upsample, a.prologue, vd._dt(x), od, a.nchw, True, a.impl)
+    d = vd.conv_desc(a.batch, a.h, a.w, a.cin, a.cout, a.k, (2 if a.phase else 1) if a.upsample else 0, a.prologue, vd._dt(x), od, a.nchw, True, a.impl)
     nb = ctypes.c_size_t(0)
     vd._check(vd.lib().vd_conv_packed_weight_bytes(ctypes.byref(d), ctypes.byref(nb)))
     packed = torch.empty(nb.value, dtype=torch.uint8, device="cuda")

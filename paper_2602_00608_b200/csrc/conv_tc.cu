@@ -34,6 +34,7 @@
 //     see TileCfg).
 // Every wait is bounded: on expiry the CTA records a code in the status word and unwinds.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -52,7 +53,7 @@ namespace {
 using namespace tc;
 using namespace convtile;
 
-constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 4;
+constexpr int MAX_B_STAGES = 8, MAX_A_STAGES = 6;
 constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epilogue warp's share of an output slice
 
 // BN = output channels per work item.  Where the channel block is narrow (BN <= 128) a work
@@ -79,6 +80,14 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // is drained as soon as its last tap has completed, while the MMAs of the other parities go on.
 // A weight stage holds the two column taps (dx = 0, 1) of one (parity, dy): 8 MMAs per stage, so
 // the issue sequence per stage is as long as that of the other forms.
+// With four accumulators and no spare set, an accumulator is needed again right after its item's last
+// chunk, and draining it takes about as long as a chunk's MMAs.  So the parities are staggered (where
+// the input has at least four chunks): parity p works on the chunk that came p chunks earlier, the four
+// accumulators complete one chunk apart, and within a chunk slot the parities run in a rotating order in
+// which the one that completes goes first and the one that completed a slot before goes last: between an
+// accumulator's last MMA and its next first MMA lie the MMAs of six (parity, chunk) blocks.  An operand
+// chunk therefore stays in shared memory for four slots (five stages).  PhaseSched is that schedule; the
+// weight loader follows it step by step.
 template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static_assert(CG == 1 || BN == 256 || PH, "the two-CTA form exists for 256-channel blocks and the phase form");
     static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
@@ -86,9 +95,9 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static constexpr int B_STAGE_BYTES = (PH ? 2 : 1) * (BN / CG) * 128;   // this CTA's rows x 64 bf16 (phase: two taps)
     static constexpr int OUT_BUFS = PH ? 2 : 1;                      // output slices per epilogue warp
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
-    static constexpr int B_STAGES = PH ? 5 : (CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
+    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
-    static constexpr int A_STAGES = 2;
+    static constexpr int A_STAGES = PH ? 5 : 2;                    // phase form: a chunk stays until the parity that lags most has used it
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
     static constexpr int SMEM_B = (B_STAGES * B_STAGE_BYTES + 1023) / 1024 * 1024;
     static constexpr int SMEM_OUT = BN >= 128 ? OUT_BUFS * OUT_SLICE_BYTES : 0;       // output slice(s) per epilogue warp
@@ -96,7 +105,7 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static constexpr int SMEM_BIAS = BN >= 128 ? 4 * BN * 4 : 0;     // one bias copy per epilogue warp
     static constexpr int SMEM_BARS = 512;
     // two-tile items and two-CTA pairs: the producers stage the raw input of the next unit in shared memory (cp.async)
-    static constexpr bool STAGED = PAIR == 2 || CG == 2;
+    static constexpr bool STAGED = !PH && (PAIR == 2 || CG == 2);
     static constexpr int SMEM_RAW = STAGED ? ITEMS * 32 : 0;
     static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + SMEM_BARS + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
@@ -148,6 +157,21 @@ struct Sched {
     __device__ __forceinline__ int index(int t, int s) const { return cg == 2 ? t + rank : t + s; }
 };
 
+// The phase form's order of (parity, chunk) blocks.  The CTA's work is a sequence of chunk slots
+// q = item * K + chunk (K chunks per item); in step s the parities run in the order (r + j) & 3, j = 0..3, and
+// parity p works on slot q = s - p * lag (skipped while that is outside [0, S)).
+struct PhaseSched {
+    int K, S, lag;
+    uint32_t m_k;                // ceil(2^32 / K), 0 for K = 1
+    __device__ __forceinline__ void init(int kchunks, int nitems) {
+        K = kchunks; S = nitems * kchunks; lag = kchunks >= 4 ? 1 : 0;
+        m_k = K == 1 ? 0u : (uint32_t)((0x100000000ull + (uint32_t)K - 1) / (uint32_t)K);
+    }
+    __device__ __forceinline__ int steps() const { return S + 3 * lag; }
+    __device__ __forceinline__ int rot(int s) const { return lag ? ((s + 1 + 3 * K) & 3) : 0; }
+    __device__ __forceinline__ int item_of(int q) const { return m_k ? (int)__umulhi((uint32_t)q, m_k) : q; }
+};
+
 // ---- cluster / cta_group::2 PTX
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -161,6 +185,9 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t cta)
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
@@ -563,7 +590,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                     load_raw_at(false, xb + (((int)(pyx[u] & 0xffu) - 1) * a.W + ((int)((pyx[u] >> 8) & 0xffu) - 1)) * a.Cin2 * 4, raw[u]);
                         }
                         if (slot == 0) {
-                            ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
+                            ok = mbar_wait<PH ? 256 : 0>(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                             if (!ok) break;
                         }
                         uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + slot * A_TILE_BYTES;
@@ -583,7 +610,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                         for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], tanh_fast(v[e]), v[e]);
                                     }
                                 }
-                                o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]);
+                                // phase form: fp16 operands (see pack_weight_phase_kernel); out-of-range values saturate
+                                if (PH) { o0 = pack_f16(v[0], v[1]); o1 = pack_f16(v[2], v[3]); o2 = pack_f16(v[4], v[5]); o3 = pack_f16(v[6], v[7]); }
+                                else { o0 = pack_bf16(v[0], v[1]); o1 = pack_bf16(v[2], v[3]); o2 = pack_bf16(v[4], v[5]); o3 = pack_bf16(v[6], v[7]); }
                             }
                             if (in_bf16) {
                                 *(uint4*)(dst_tile + soff[u]) = make_uint4(o0, o1, o2, o3);
@@ -706,14 +735,20 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     const uint32_t tacc = tmem_base + (uint32_t)((buf * PAIR + slot) * Cfg::ACC_COLS) + ((uint32_t)(ew * 32) << 16);
                     const bool last_tile = PH || slot == cnt - 1;
                     const int acc_bar = PH ? slot : buf;
+                    // A TMEM read queues behind the MMAs already issued (measured: its latency grows with the number of
+                    // weight stages the MMA warp is ahead), so the round trips are what a drain costs.  Where the drain
+                    // is on the critical path (phase form: no second accumulator set) two passes are read per round trip;
+                    // elsewhere the next pass is in flight while one is processed.
+                    constexpr bool PAIRED = PH;
                     uint32_t ra[32], rb[32];
                     tmem_ld32(tacc, ra);
+                    if (PAIRED) tmem_ld32(tacc + 32u, rb);
                     tmem_ld_wait();
 #pragma unroll
                     for (int p = 0; p < NP; ++p) {
                         uint32_t (&rc)[32] = (p & 1) ? rb : ra;          // this pass
                         uint32_t (&rn)[32] = (p & 1) ? ra : rb;          // next pass, in flight while this one is processed
-                        if (p + 1 < NP) tmem_ld32(tacc + (uint32_t)((p + 1) * 32), rn);
+                        if (!PAIRED && p + 1 < NP) tmem_ld32(tacc + (uint32_t)((p + 1) * 32), rn);
                         const int sl = p / PPS, h = p % PPS;              // slice, half of the slice
                         // The CTA's last item has the weight stages to itself (every MMA has completed): its slices go
                         // through a longer ring of buffers there, so the stores of the tail are not paced by buffer reuse.
@@ -747,12 +782,22 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                                pack_bf16(__uint_as_float(rc[8 * c + 6]) + t1.z, __uint_as_float(rc[8 * c + 7]) + t1.w));
                             }
                         }
+                        if (PAIRED && (p & 1) && p + 1 < NP) {           // both buffers are free again: the next two passes
+                            tmem_ld32(tacc + (uint32_t)((p + 1) * 32), ra);
+                            tmem_ld32(tacc + (uint32_t)((p + 2) * 32), rb);
+                        }
                         if (p + 1 < NP) {
-                            tmem_ld_wait();
-                        } else if (last_tile) {                          // accumulators fully read: hand them back
+                            if (!PAIRED || (p & 1)) tmem_ld_wait();
+                        }
+                        // accumulators fully read (the last read has landed in registers): hand them back.  The arrival
+                        // carries no data (the reads are complete), so it need not wait for this warp's shared-memory stores.
+                        if (last_tile && (PAIRED ? p == NP - 3 : p == NP - 1)) {
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) arrive_leader(&bars->acc_empty[acc_bar]);
+                            if (lane == 0) {
+                                if (PAIRED && CG == 2) mbar_arrive_cluster_relaxed(map_to_cta(smem_u32(&bars->acc_empty[acc_bar]), 0));
+                                else arrive_leader(&bars->acc_empty[acc_bar]);
+                            }
                         }
                         if (h == PPS - 1) {
                             fence_proxy_async_smem();
@@ -848,24 +893,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             bool ok = true;
             for (int t = sched.begin; t < sched.end && ok; t += sched.count(t)) {
                 const Tile tl = sched.get(t, BN);
-                if constexpr (PH) {
-                    // eight stages per chunk: (parity, dy), each with the taps dx = 0, 1 of this CTA's 64 output
-                    // channels as one box of 128 rows (the packed layout keeps them adjacent)
-                    const int blk = tl.n0 / BN;
-                    for (int kc = 0; kc < kchunks && ok; ++kc) {
-                        for (int st = 0; st < 8; ++st) {
-                            ok = mbar_wait(smem_u32(&bars->b_empty[stage]), phase ^ 1, abort_flag);
-                            if (!ok) break;
-                            const uint32_t dst = smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES);
-                            const uint32_t full = leader_bar(&bars->b_full[stage]);
-                            mbar_arrive_expect_tx_cluster(full, Cfg::B_STAGE_BYTES);
-                            tma_load_2d_pair(dst, &tmap, kc * 64, ((st * sched.nblk + blk) * 2 + (int)rank) * 128, full);
-                            ++issued;
-                            if (++stage == Cfg::B_STAGES) { stage = 0; phase ^= 1; }
-                        }
-                    }
-                    continue;
-                }
+                if constexpr (PH) break;                 // the phase form streams its weights in PhaseSched order, below
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
                     const bool second = kc >= kchunks;
                     const int ntap = second ? 1 : taps;
@@ -892,6 +920,37 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     }
                 }
             }
+            if constexpr (PH) {
+                // two stages per (parity, chunk) block: dy = 0, 1, each with the taps dx = 0, 1 of this CTA's 64
+                // output channels as one box of 128 rows (the packed layout keeps them adjacent)
+                int nitems = 0;
+                for (int t = sched.begin; t < sched.end; t += sched.count(t)) ++nitems;
+                PhaseSched ps; ps.init(kchunks, nitems);
+                int blk_of[2] = {0, 0};                      // channel block of the item (index & 1)
+                int t_next = sched.begin;
+                for (int s = 0; s < ps.steps() && ok; ++s) {
+                    if (s < ps.S && s == ps.item_of(s) * ps.K) {         // a new item starts in this step
+                        blk_of[ps.item_of(s) & 1] = sched.get(t_next, BN).n0 / BN;
+                        t_next += sched.count(t_next);
+                    }
+                    const int r = ps.rot(s);
+                    for (int j = 0; j < 4 && ok; ++j) {
+                        const int p = (r + j) & 3, q = s - p * ps.lag;
+                        if (q < 0 || q >= ps.S) continue;
+                        const int it = ps.item_of(q), kc = q - it * ps.K;
+                        for (int dy = 0; dy < 2; ++dy) {
+                            ok = mbar_wait(smem_u32(&bars->b_empty[stage]), phase ^ 1, abort_flag);
+                            if (!ok) break;
+                            const uint32_t dst = smem_u32(smem_b + stage * Cfg::B_STAGE_BYTES);
+                            const uint32_t full = leader_bar(&bars->b_full[stage]);
+                            mbar_arrive_expect_tx_cluster(full, Cfg::B_STAGE_BYTES);
+                            tma_load_2d_pair(dst, &tmap, kc * 64, (((2 * p + dy) * sched.nblk + blk_of[it & 1]) * 2 + (int)rank) * 128, full);
+                            ++issued;
+                            if (++stage == Cfg::B_STAGES) { stage = 0; phase ^= 1; }
+                        }
+                    }
+                }
+            }
             if (!ok) {
                 // unwinding: let the copies already in flight land before the CTA's memory is released
                 uint32_t s = stage, ph = phase;
@@ -912,7 +971,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         // is two tiles the warp issues for both.
         {
             const bool leader = elect_one() != 0u;
-            constexpr uint32_t idesc = make_idesc_bf16(128 * CG, BN);
+            constexpr uint32_t idesc = PH ? make_idesc_f16(128 * CG, BN) : make_idesc_bf16(128 * CG, BN);
             const uint32_t a_hi = desc_hi(PW * 128, 2), b_hi = desc_hi(1024, 2);
             const uint32_t a_lo0 = desc_lo(smem_u32(smem_a)), b_lo0 = desc_lo(smem_u32(smem_b));
             // one MMA of the pair (M = 256 over both CTAs) or of this CTA; a commit to both CTAs or to this one
@@ -998,24 +1057,33 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     commit_on(smem_u32(&bars->acc_full[buf]));
                     __syncwarp();
                 };
-                // phase form: per chunk, the four parities' 2 x 2 taps (see TileCfg); parity p = 2a + b accumulates
-                // in columns [128p, 128p + 128), waits for its own "empty" barrier before the item's first tap and
-                // reports "full" after its last, so the epilogue drains parity 0 while parities 1..3 still compute
-                auto item_phase = [&](int n_it) {
+                // phase form: (parity, chunk) blocks in PhaseSched order.  Parity p = 2a + b accumulates in columns
+                // [128p, 128p + 128), waits for its own "empty" barrier before an item's first chunk and reports
+                // "full" after its last; an operand stage goes back once parity 3 (which lags most) has used it
+                if constexpr (PH) {
+                    int nitems = 0;
+                    for (int t = sched.begin; t < sched.end; t += sched.count(t)) ++nitems;
+                    PhaseSched ps; ps.init(kchunks, nitems);
 #pragma unroll 1
-                    for (int kc = 0; kc < kchunks; ++kc) {
-                        const bool first = kc == 0, last = kc == kchunks - 1;
-                        wait_on(smem_u32(&bars->a_full[as]), aph);
-                        const uint32_t a_base = a_lo0 + as * (A_STAGE_BYTES >> 4);
-#pragma unroll
-                        for (int p = 0; p < 4; ++p) {
+                    for (int s = 0; s < ps.steps(); ++s) {
+                        if (*abort_flag) break;
+                        const int r = ps.rot(s);
+#pragma unroll 1
+                        for (int j = 0; j < 4; ++j) {
+                            const int p = (r + j) & 3, q = s - p * ps.lag;
+                            if (q < 0 || q >= ps.S) continue;
+                            const int it = ps.item_of(q), kc = q - it * ps.K;
+                            const uint32_t st = (uint32_t)q % (uint32_t)Cfg::A_STAGES;
+                            if (p == 0) wait_on(smem_u32(&bars->a_full[st]), ((uint32_t)q / (uint32_t)Cfg::A_STAGES) & 1u);
+                            const bool first = kc == 0, last = kc == ps.K - 1;
+                            if (first) wait_on(smem_u32(&bars->acc_empty[p]), (uint32_t)((it & 1) ^ 1));
                             const uint32_t td = tmem_base + (uint32_t)(p * Cfg::ACC_COLS);
-                            if (first) wait_on(smem_u32(&bars->acc_empty[p]), (uint32_t)((n_it & 1) ^ 1));
+                            const uint32_t a_view = a_lo0 + st * (uint32_t)(A_STAGE_BYTES >> 4) + (uint32_t)(((p >> 1) * PW + (p & 1)) * 8);
 #pragma unroll
                             for (int dy = 0; dy < 2; ++dy) {
                                 wait_on(b_full0 + bs * 8u, bph);
                                 const uint32_t b_lo = b_lo0 + bs * (uint32_t)(Cfg::B_STAGE_BYTES >> 4);
-                                const uint32_t a_lo = a_base + (uint32_t)((((p >> 1) + dy) * PW + (p & 1)) * 8);
+                                const uint32_t a_lo = a_view + (uint32_t)(dy * PW * 8);
                                 mma_on(td, a_lo, b_lo, (first && dy == 0) ? 0u : 1u);
                                 mma_on(td, a_lo + 2, b_lo + 2, 1u);
                                 mma_on(td, a_lo + 4, b_lo + 4, 1u);
@@ -1033,20 +1101,15 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 commit_on(smem_u32(&bars->acc_full[p]));
                                 __syncwarp();
                             }
+                            if (p == 3) {
+                                commit_on(smem_u32(&bars->a_empty[st]));
+                                __syncwarp();
+                            }
                         }
-                        commit_on(smem_u32(&bars->a_empty[as]));
-                        __syncwarp();
-                        if (++as == Cfg::A_STAGES) { as = 0; aph ^= 1; }
                     }
-                };
+                } else
                 for (int t = sched.begin; t < sched.end; ++n_item) {
                     const int n = sched.count(t);
-                    if constexpr (PH) {
-                        if (*abort_flag) break;
-                        item_phase(n_item);
-                        t += n;
-                        continue;
-                    }
                     const int buf = n_item % NBUF;
                     wait_on(smem_u32(&bars->acc_empty[buf]), ((n_item / NBUF) & 1) ^ 1);
                     if (*abort_flag) break;
@@ -1160,9 +1223,15 @@ __global__ void pack_weight_tc_kernel(const T* w, __nv_bfloat16* packed, int Cou
 // column taps of one (parity, dy) for one CTA's half of a channel block are one box of 128 rows.
 // The weight at (parity (a, b), dy, dx) is the sum of the 3x3 taps (ky, kx) that read the same source
 // pixel: a = 0: dy 0 <- ky {0}, dy 1 <- ky {1, 2};  a = 1: dy 0 <- ky {0, 1}, dy 1 <- ky {2};  columns alike.
-// The sum is formed in fp32 in a fixed order and rounded once to bf16.
+// The sum is formed in fp32 in a fixed order and rounded once, to FP16, and the kernel converts the
+// activation operand of these layers to fp16 as well (same tensor rate as bf16): a sum of up to four bf16
+// weights is not a bf16 number, and rounding it to bf16 would add a second 2^-9 error per product to these
+// layers; fp16 rounds both operands eight times finer instead (magnitudes are far inside its range: weights
+// below 1, activations saturate at 65504; a sum below 2^-14 is rounded with an absolute error of at most 2^-25).
+// Both operands of one tcgen05.mma kind::f16 must have the same format: fp16 weights beside bf16 activations
+// are an illegal instruction on this device.
 template <typename T>
-__global__ void pack_weight_phase_kernel(const T* w, __nv_bfloat16* packed, int Cout, int Cin) {
+__global__ void pack_weight_phase_kernel(const T* w, __half* packed, int Cout, int Cin) {
     const int64_t total = (int64_t)16 * Cout * Cin;
     const int nblk = Cout / 128;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -1181,7 +1250,7 @@ __global__ void pack_weight_phase_kernel(const T* w, __nv_bfloat16* packed, int 
             }
         const int st = par * 2 + dy, blk = o / 128, rk = (o % 128) / 64, r = o % 64;
         const size_t row = ((((size_t)st * nblk + blk) * 2 + rk) * 2 + dx) * 64 + r;
-        packed[row * Cin + c] = __float2bfloat16_rn(v);
+        packed[row * Cin + c] = __float2half_rn(v);
     }
 }
 
@@ -1343,8 +1412,8 @@ cudaError_t launch_pack_weight_tc(const void* w, int w_dtype, void* packed, int 
         if (taps != 9 || cout_offset != 0 || cout_total != Cout || Cout % 128 != 0) return cudaErrorInvalidValue;
         const int64_t n = (int64_t)16 * Cout * Cin;
         const int grid = (int)std::min<int64_t>((n + 255) / 256, 148 * 16);
-        if (w_dtype == VD_BF16) pack_weight_phase_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)w, (__nv_bfloat16*)packed, Cout, Cin);
-        else pack_weight_phase_kernel<float><<<grid, 256, 0, s>>>((const float*)w, (__nv_bfloat16*)packed, Cout, Cin);
+        if (w_dtype == VD_BF16) pack_weight_phase_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)w, (__half*)packed, Cout, Cin);
+        else pack_weight_phase_kernel<float><<<grid, 256, 0, s>>>((const float*)w, (__half*)packed, Cout, Cin);
         return cudaGetLastError();
     }
     const int cpad = padded_cout(cout_total);

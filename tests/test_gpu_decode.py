@@ -145,7 +145,8 @@ def test_full_size_configs_whole_frame_against_the_oracle(env, idx):
     d = (a - got2.float())
     r2 = float(d.norm() / got2.float().norm())
     print(f"tcgen05 vs FFMA {wl.name}: rel-L2 {r2:.3e} max-abs {float(d.abs().max()):.3e}")
-    assert r2 <= 6e-3 and float(d.abs().max()) <= BF16_MAX_ABS
+    # two independently rounded bf16 runs differ by about sqrt(2) x the error of one against fp32 math
+    assert r2 <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
 
 
 def test_host_buffer_decode_and_extrapolation(env):

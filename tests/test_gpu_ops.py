@@ -245,14 +245,14 @@ def test_conv_tc_phase_collapsed_upsample_matches_oracle(env, case):
     _, _, vd, _ = env
     got, want = _conv_case(env, seed=47, impl=vd.VD_IMPL_TC, bf16_ops=True, **case)
     assert got.shape == want.shape
-    # as test_conv_tc_matches_oracle, plus one bf16 rounding of every pre-summed weight (another
-    # 2^-9 relative per product, independent of the operand's): sqrt(2) x the one-rounding error
-    tol = 4.5e-3 if case["out_bf16"] else 3e-3
+    # both operands of this form are fp16 (2^-12 relative per rounding, activations and pre-summed
+    # weights alike): an eighth of the bf16 forms' error; a bf16 output adds its own 2^-9 rounding
+    tol = 4e-3 if case["out_bf16"] else 6e-4
     assert rel_l2(got, want) <= tol
     # against the 9-tap folded form of the same kernel family: same operands, weights summed after
     # instead of before the rounding
     got9, _ = _conv_case(env, seed=47, impl=vd.VD_IMPL_TC, bf16_ops=True, **dict(case, upsample=1))
-    assert rel_l2(got, got9) <= (4.5e-3 if case["out_bf16"] else 2e-3)
+    assert rel_l2(got, got9) <= (4.5e-3 if case["out_bf16"] else 2.5e-3)
 
 
 @pytest.mark.parametrize("ky,kx", [(ky, kx) for ky in range(3) for kx in range(3)])
@@ -263,6 +263,7 @@ def test_conv_tc_phase_collapsed_single_taps_are_exact(env, ky, kx):
     torch, ref, vd, synth = env
     B, H, W, C = 2, 19, 10, 64
     x = synth.round_to_bf16(_rng(7).standard_normal((B, C, H, W)).astype(np.float32))
+    x[np.abs(x) < 2.0 ** -10] = 0.0       # the kernel's operands are fp16: bf16 values this small would not convert exactly
     w = np.zeros((128, C, 3, 3), np.float32)
     w[np.arange(C), np.arange(C), ky, kx] = 1.0
     y = vd.op_conv2d(util.nchw_to_dev_nhwc(x, torch.bfloat16), torch.from_numpy(w).cuda().bfloat16(),
