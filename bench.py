@@ -36,11 +36,18 @@ def load_peaks():
     return d
 
 
-def contract_roofline_us(steps, peaks, batch, stream_bytes=2):
+def executed_flops(s):
+    """Flops the kernel of a step executes: a phase-collapsed upsampling convolution issues 4 of the 9 taps."""
+    return s["flops_per_frame"] * (4.0 / 9.0 if s.get("phase_collapsed") else 1.0)
+
+
+def contract_roofline_us(steps, peaks, batch, stream_bytes=2, four_tap=False):
     """Per-layer roofline of one frame: sum over layers of max(flops/peak, bytes/HBM).  Bytes are
     the algorithmic ones (input once at source resolution, residual once, output once, weights
     once per batch) with every activation counted at `stream_bytes` (2 = bf16 everywhere, the
-    contract denominator) or as stored (stream_bytes=None)."""
+    contract denominator) or as stored (stream_bytes=None).  Flops are the layers' own (9 taps on
+    the upsampled grid for an upsampling convolution); four_tap=True counts the phase-collapsed
+    layers at the 4 taps they execute (the stricter denominator)."""
     tf = peaks["bf16_tflops"] * 1e12
     bw = peaks["hbm_gbs"] * 1e9
     total = 0.0
@@ -49,7 +56,7 @@ def contract_roofline_us(steps, peaks, batch, stream_bytes=2):
     for s in steps:
         if s["kind"] == 0:
             continue
-        fl = s["flops_per_frame"]
+        fl = executed_flops(s) if four_tap else s["flops_per_frame"]
         if stream_bytes is None:
             by = s["bytes_per_frame"]
         else:
@@ -202,6 +209,15 @@ def main():
 
     from paper_2602_00608_b200 import synth
     wl = synth.WORKLOADS[args.config]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly with --gpus N: run N replicas, one rank per GPU, under torchrun
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -256,16 +272,29 @@ def main():
                     break
             except OSError:
                 break
-    barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_region(fn, steps):
+        """EXACTLY `steps` calls of fn between barrier + synchronize on both sides; device time, max over ranks."""
+        barrier()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1))
+
+    def timed_regions(fn, steps):
+        """Regions of `steps` calls back to back until about a second of load has been timed (at least
+        five), so that the clock record holds enough samples; the median region is the reported one."""
+        first = timed_region(fn, steps)
+        n = max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1))
+        return [first] + [timed_region(fn, steps) for _ in range(n - 1)]
+
     t_begin = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        dec.decode(z, frames)
-    e1.record(stream)
-    barrier()
+    regions = timed_regions(lambda: dec.decode(z, frames), args.steps)
     t_end = time.time()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = sorted(regions)[len(regions) // 2]
     dec.check_status()
     clocks = sampler.stop(t_begin, t_end) if sampler else None
     ms_step = ms_total / args.steps
@@ -274,18 +303,20 @@ def main():
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
     zh = torch.from_numpy(z_np).to(dec.dtype).pin_memory()
     fh = torch.empty((wl.batch,) + dec.out_shape, dtype=dec.dtype).pin_memory()
-    e2e_steps = max(3, min(args.steps, 10))
     dec.decode_host(zh, fh)
-    barrier()
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        dec.decode_host(zh, fh)
-    e1.record(stream)
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    sampler2 = ClockSampler(local_rank) if rank == 0 else None
+    if sampler2:
+        sampler2.wait_for_samples(1)
+    t2_begin = time.time()
+    e2e_regions = timed_regions(lambda: dec.decode_host(zh, fh), args.steps)
+    t2_end = time.time()
+    e2e_clocks = sampler2.stop(t2_begin, t2_end) if sampler2 else None
+    e2e_ms = sorted(e2e_regions)[len(e2e_regions) // 2] / args.steps
     e2e = {"value": replicas.whole_job_rate(world, wl.batch, 1, e2e_ms), "unit": "frames/s",
            "h2d_bytes_per_step": zh.numel() * zh.element_size(), "d2h_bytes_per_step": fh.numel() * fh.element_size(),
-           "ms_per_step": e2e_ms}
+           "ms_per_step": e2e_ms, "ms_per_step_best": min(e2e_regions) / args.steps, "regions": len(e2e_regions),
+           "api": "vd_decode_host (pinned host buffers; H2D copy, decode, D2H copy and stream synchronise per step)",
+           "clocks": e2e_clocks}
 
     # ---- the same decode without the power cap: ten decodes after the GPU has idled for 0.2 s (the long run above
     # settles at the cap within some 20 decodes; this figure is context, `value` stays the sustained one)
@@ -321,28 +352,40 @@ def main():
         d = by_kind.setdefault(key, {"ms": 0.0, "flops": 0.0, "bytes": 0.0, "launches": 0})
         d["ms"] += ms
         d["flops"] += s["flops_per_frame"] * wl.batch
+        d["flops_exec"] = d.get("flops_exec", 0.0) + executed_flops(s) * wl.batch
         d["bytes"] += s["bytes_per_frame"] * wl.batch + s["weight_bytes"]
         d["launches"] += s["launches"]
     dom = max(by_kind, key=lambda k: by_kind[k]["ms"])
     d = by_kind[dom]
-    peak_tf = peaks["bf16_tflops_sustained"]
     if d["flops"] > 0:
-        roof = {"kernel": dom, "bound": "tensor", "achieved": d["flops"] / (d["ms"] * 1e-3) / 1e12, "peak": peak_tf,
-                "unit": "TFLOP/s", "peak_source": f"{peaks['source']} (sustained: kernel timed inside a long step)",
+        # the per-kernel times come from short profiled decodes (events around every launch, ten decodes): the
+        # burst regime, so the burst GEMM peak is the denominator; the fraction of the sustained peak is beside it
+        ach = d["flops"] / (d["ms"] * 1e-3) / 1e12
+        roof = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "peak_source": f"{peaks['source']} (burst: kernels timed one by one in short profiled decodes)",
+                "frac": ach / peaks["bf16_tflops"], "frac_burst": ach / peaks["bf16_tflops"],
+                "frac_sustained": ach / peaks["bf16_tflops_sustained"], "peak_sustained": peaks["bf16_tflops_sustained"],
+                "achieved_note": "algorithmic flops (9 taps for every 3x3 layer) / summed launch durations",
+                "achieved_executed": d["flops_exec"] / (d["ms"] * 1e-3) / 1e12,
+                "achieved_executed_note": "the same with the phase-collapsed upsampling layers counted at the 4 taps they execute",
                 "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get((wl.name, dom)), "traffic_unit": "bytes per launch (ncu, cold cache)",
                 "launches_per_step": d["launches"], "ms_per_step": d["ms"]}
     else:
-        roof = {"kernel": dom, "bound": "hbm", "achieved": d["bytes"] / (d["ms"] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "peak_source": peaks["source"], "traffic": None, "launches_per_step": d["launches"],
-                "ms_per_step": d["ms"]}
-    roof["frac"] = roof["achieved"] / roof["peak"]
+        ach = d["bytes"] / (d["ms"] * 1e-3) / 1e9
+        roof = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "peak_source": peaks["source"], "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                "launches_per_step": d["launches"], "ms_per_step": d["ms"]}
     gn = by_kind.get("gn_stats")
     contract_us, flops_frame, bytes_frame = contract_roofline_us(steps, peaks, wl.batch, 2)
     stored_us, _, stored_bytes = contract_roofline_us(steps, peaks, wl.batch, None)
     per_frame_us = ms_step * 1e3 / wl.batch
+    four_us, four_flops, _ = contract_roofline_us(steps, peaks, wl.batch, 2, four_tap=True)
     decoder_roofline = {
         "per_layer_roofline_us_per_frame": contract_us, "measured_us_per_frame": per_frame_us,
-        "frac": contract_us / per_frame_us, "gflop_per_frame": flops_frame / 1e9, "gbytes_per_frame": bytes_frame / 1e9,
+        "frac": contract_us / per_frame_us,
+        # stricter denominator: the upsampling convolutions counted at the 4 taps the phase-collapsed form executes
+        "four_tap_roofline_us_per_frame": four_us, "frac_four_tap": four_us / per_frame_us, "gflop_per_frame_four_tap": four_flops / 1e9,
+        "regions": len(regions), "ms_per_step_best": min(regions) / args.steps, "gflop_per_frame": flops_frame / 1e9, "gbytes_per_frame": bytes_frame / 1e9,
         "as_stored_roofline_us_per_frame": stored_us, "as_stored_frac": stored_us / per_frame_us,
         "as_stored_gbytes_per_frame": stored_bytes / 1e9,
         # the timed region is a long, power-capped run: the same per-layer sum with the GEMM peak measured in that
@@ -361,6 +404,21 @@ def main():
             dist.destroy_process_group()
         return
 
+    # parity of what was just timed: the last frame of the batch against the oracle's frame for the same seeded
+    # latents (stored by tests/golden/make_golden.py --full, which calls only the oracle), every pixel
+    parity = None
+    gold_path = os.path.join(ROOT, "tests", "golden", f"frame_cfg{args.config}_full.npz")
+    if os.path.exists(gold_path) and not args.simt:
+        import numpy as np
+        gold = np.load(gold_path)
+        dec.decode(z, frames)
+        torch.cuda.synchronize()
+        g = frames[int(gold["index"])].float().cpu().numpy().astype(np.float64)
+        w = gold["frame"].astype(np.float64)
+        parity = {"rel_l2": float(np.linalg.norm(g - w) / np.linalg.norm(w)), "max_abs": float(np.abs(g - w).max()),
+                  "frame": int(gold["index"]), "pixels": int(w.size), "bar": {"rel_l2": 1e-2, "max_abs": 3e-2},
+                  "against": "oracle frame, every pixel (tests/golden, written by the oracle alone)"}
+
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
         cpu_baseline, _ = time_oracle(wl, 2, 1, 0)
@@ -370,14 +428,14 @@ def main():
         "metric": "720x480 decoded frames/s on 1 B200 (bf16); % of per-layer roofline" if args.config in (3, 4)
                   else f"decoded frames/s ({wl.out_w}x{wl.out_h})",
         "value": fps, "unit": "frames/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_step, "timing": f"median of {len(regions)} back-to-back regions of {args.steps} steps", "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": wl.name, "batch": wl.batch, "latent": [wl.latent_h, wl.latent_w],
                    "frame": [wl.out_h, wl.out_w], "parallelism": f"replicas x{world}",
                    "l2": "no flush: each step streams several GB of activations, far beyond the 126 MB L2",
                    "kernels": "ffma" if args.simt else "tcgen05+ffma"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roof,
-        "decoder_roofline": decoder_roofline, "cpu_baseline": cpu_baseline,
+        "decoder_roofline": decoder_roofline, "parity": parity, "cpu_baseline": cpu_baseline,
         "paper_context": "paper reports 109.4 ms per 720x480 frame (9.1 frames/s) for its fused decoder on one Ascend 910C (Table II)",
     }
     print(json.dumps(line), flush=True)
