@@ -63,6 +63,7 @@ def lib():
             l.vd_ref_add.argtypes = [_f32p, _f32p, _f32p, lg]
             l.vd_ref_attention_core.argtypes = [_f32p, _f32p, _f32p, _f32p, i, i, i, f, _f64p]
             l.vd_ref_extrapolate.argtypes = [_f32p, _f32p, f, _f32p, _f32p, lg]
+            l.vd_ref_pack_u8.argtypes = [_f32p, ctypes.POINTER(ctypes.c_ubyte), i, i, i, i]
             _lib = l
     return _lib
 
@@ -155,6 +156,16 @@ def extrapolate(z_prev, v_prev, lam: float):
     v = np.empty_like(z_prev)
     _ok(lib().vd_ref_extrapolate(_p(z_prev), _p(v_prev), lam, _p(z), _p(v), z_prev.size), "extrapolate")
     return z, v
+
+
+def pack_u8(x):
+    """Display packing of frames for transport (output side of Algorithm 1's decode step): NCHW fp32 in
+    [-1, 1] -> NHWC uint8, q = rint(clamp(fma(x, 127.5, 127.5), 0, 255)) in fp32, ties to even."""
+    x = _c(x)
+    n, c, h, w = x.shape
+    q = np.empty((n, h, w, c), np.uint8)
+    _ok(lib().vd_ref_pack_u8(_p(x), q.ctypes.data_as(ctypes.POINTER(ctypes.c_ubyte)), n, c, h, w), "pack_u8")
+    return q
 
 
 # ---------------------------------------------------------------------------------------------

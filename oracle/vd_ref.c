@@ -234,3 +234,27 @@ VD_REF_API int vd_ref_extrapolate(const float* z_prev, const float* v_prev, floa
     }
     return 0;
 }
+
+/*
+ * Display packing of a decoded frame for transport to the host (the output side of the decode step of
+ * Algorithm 1, Q_out.push(I_t); Table II lists the frame transport as a component of its own).  The
+ * paper does not print the mapping; the reading taken is the usual one for a decoder whose frames live in
+ * [-1, 1]: q = round(clamp(x * 0.5 + 0.5, 0, 1) * 255), channels interleaved per pixel (NHWC), 8 bits.
+ * A floating-point value decides an integer here, so the arithmetic is fixed to what the kernels do, in
+ * fp32: t = fma(x, 127.5, 127.5) (one rounding), clamped to [0, 255], rounded to nearest with ties to
+ * even.  NaN packs to 0.
+ *   x: [N,C,H,W] fp32     q: [N,H,W,C] uint8
+ */
+VD_REF_API int vd_ref_pack_u8(const float* x, unsigned char* q, int N, int C, int H, int W) {
+    if (!x || !q || N < 0 || C <= 0 || H <= 0 || W <= 0) return -1;
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int i = 0; i < H; ++i)
+                for (int j = 0; j < W; ++j) {
+                    float t = fmaf(x[(((size_t)n * C + c) * H + i) * W + j], 127.5f, 127.5f);
+                    if (!(t > 0.0f)) t = 0.0f;              /* also NaN */
+                    if (t > 255.0f) t = 255.0f;
+                    q[(((size_t)n * H + i) * W + j) * C + c] = (unsigned char)rintf(t);
+                }
+    return 0;
+}

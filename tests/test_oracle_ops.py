@@ -274,3 +274,35 @@ def test_results_do_not_depend_on_thread_count():
         assert np.array_equal(ref.conv2d(x, w), y_many)
     finally:
         ref.set_num_threads(n)
+
+
+def test_pack_u8_fixed_points_saturation_and_layout():
+    # -1 -> 0, 0 -> 128 (127.5 ties to even), 1 -> 255; anything outside saturates; NaN -> 0
+    x = np.array([-1.0, 0.0, 1.0, -7.0, 3.0, np.nan, -1e30, 1e30], np.float32).reshape(1, 1, 2, 4)
+    assert ref.pack_u8(x).ravel().tolist() == [0, 128, 255, 0, 255, 0, 0, 255]
+    # channel interleaving: [N,C,H,W] -> [N,H,W,C]
+    y = np.stack([np.full((2, 3), -1.0), np.zeros((2, 3)), np.ones((2, 3))]).astype(np.float32)[None]
+    q = ref.pack_u8(y)
+    assert q.shape == (1, 2, 3, 3) and (q[0, :, :, 0] == 0).all() and (q[0, :, :, 1] == 128).all() and (q[0, :, :, 2] == 255).all()
+
+
+def test_pack_u8_is_the_exact_rounding_away_from_boundaries_and_monotone():
+    from fractions import Fraction
+    r = np.random.Generator(np.random.Philox(key=71))
+    x = np.sort(np.concatenate([r.uniform(-1.2, 1.2, 4000), np.linspace(-1, 1, 511)]).astype(np.float32))
+    q = ref.pack_u8(x.reshape(1, 1, 1, -1)).ravel().astype(int)
+    assert (np.diff(q) >= 0).all()                                     # monotone
+    checked = 0
+    for xv, qv in zip(x.tolist(), q.tolist()):
+        t = Fraction(xv) * Fraction(255, 2) + Fraction(255, 2)         # exact x * 127.5 + 127.5
+        t = min(max(t, Fraction(0)), Fraction(255))
+        lo = int(t)                                                    # floor (t >= 0)
+        frac = t - lo
+        if abs(frac - Fraction(1, 2)) > Fraction(1, 10000):            # away from a rounding boundary: one answer
+            assert qv == (lo if frac < Fraction(1, 2) else lo + 1), (xv, qv)
+            checked += 1
+    assert checked > 4000
+    # every level is reached exactly at its centre x = (2k - 255) / 255
+    k = np.arange(256)
+    centres = ((2.0 * k - 255.0) / 255.0).astype(np.float32)
+    assert (ref.pack_u8(centres.reshape(1, 1, 1, -1)).ravel() == k).all()
