@@ -301,21 +301,43 @@ def main():
     fps = replicas.whole_job_rate(world, wl.batch, args.steps, ms_total)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
-    zh = torch.from_numpy(z_np).to(dec.dtype).pin_memory()
-    fh = torch.empty((wl.batch,) + dec.out_shape, dtype=dec.dtype).pin_memory()
-    dec.decode_host(zh, fh)
+    # A region of K steps is ceil(K / 32) calls of vd_decode_host_stream, each over up to 32 steps' worth of
+    # latents and frames in pinned host memory: every step's latents are copied in and every step's frames
+    # are copied out inside the timed region, overlapped with the neighbouring decodes.
+    chunk = min(args.steps, 32)
+    zh = torch.from_numpy(z_np).to(dec.dtype).repeat(chunk, 1, 1, 1).pin_memory()
+    fh = torch.empty((chunk * wl.batch,) + dec.out_shape, dtype=dec.dtype).pin_memory()
+    calls = [min(chunk, args.steps - i) for i in range(0, args.steps, chunk)]
+
+    def e2e_region():
+        barrier()
+        e0.record(stream)
+        for n in calls:
+            dec.decode_host_stream(zh[:n * wl.batch], fh[:n * wl.batch], batch=wl.batch)
+        e1.record(stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1))
+
+    e2e_region()
     sampler2 = ClockSampler(local_rank) if rank == 0 else None
     if sampler2:
         sampler2.wait_for_samples(1)
     t2_begin = time.time()
-    e2e_regions = timed_regions(lambda: dec.decode_host(zh, fh), args.steps)
+    first = e2e_region()
+    e2e_regions = [first] + [e2e_region() for _ in range(max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1)) - 1)]
     t2_end = time.time()
     e2e_clocks = sampler2.stop(t2_begin, t2_end) if sampler2 else None
     e2e_ms = sorted(e2e_regions)[len(e2e_regions) // 2] / args.steps
+    # the serial form for context: copy in, decode, copy out, synchronise, one step at a time
+    zh1 = zh[:wl.batch].clone().pin_memory()
+    fh1 = fh[:wl.batch].clone().pin_memory()
+    serial_ms = timed_region(lambda: dec.decode_host(zh1, fh1), args.steps) / args.steps
     e2e = {"value": replicas.whole_job_rate(world, wl.batch, 1, e2e_ms), "unit": "frames/s",
-           "h2d_bytes_per_step": zh.numel() * zh.element_size(), "d2h_bytes_per_step": fh.numel() * fh.element_size(),
+           "h2d_bytes_per_step": zh1.numel() * zh1.element_size(), "d2h_bytes_per_step": fh1.numel() * fh1.element_size(),
            "ms_per_step": e2e_ms, "ms_per_step_best": min(e2e_regions) / args.steps, "regions": len(e2e_regions),
-           "api": "vd_decode_host (pinned host buffers; H2D copy, decode, D2H copy and stream synchronise per step)",
+           "api": "vd_decode_host_stream (pinned host buffers; every step's latents copied in and frames copied out, "
+                  "overlapped with the neighbouring decodes; one host wait per call of up to 32 steps)",
+           "serial_ms_per_step": serial_ms, "serial_api": "vd_decode_host (copy in, decode, copy out, synchronise per step)",
            "clocks": e2e_clocks}
 
     # ---- the same decode without the power cap: ten decodes after the GPU has idled for 0.2 s (the long run above

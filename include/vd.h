@@ -54,6 +54,11 @@ typedef enum { VD_ARCH_TINY = 0, VD_ARCH_SDVAE = 1 } vd_arch;
 
 /* vd_config.flags */
 #define VD_FLAG_FORCE_SIMT 0x1u   /* run every layer on the plain FFMA kernels (cross-check path) */
+#define VD_FLAG_OUT_U8 0x4u       /* frames leave display-packed for transport (output side of Algorithm 1's decode
+                                     step, Q_out.push(I_t); the frame copy is Table II's "Data Transport" row): NHWC
+                                     uint8 [batch, 8*latent_h, 8*latent_w, out_channels], q = round(clamp(x*0.5+0.5,
+                                     0, 1)*255), computed in fp32 as rint(clamp(fma(x, 127.5, 127.5), 0, 255)) with ties
+                                     to even, in the last convolution's epilogue (a quarter / half of the bytes to copy) */
 #define VD_FLAG_UPSAMPLE_9TAP 0x2u /* upsampling convolutions as 9 taps on the 2x grid (upsampling folded into the
                                      addressing) instead of the default phase-collapsed form: per output parity a
                                      2x2 convolution of the source with pre-summed weights, 4/9 of the products,
@@ -104,7 +109,8 @@ VD_API vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32
 /* Decodes `batch` latents into frames (Algorithm 1, VAE decode step: I_t = Decode(z_t)).
  *   latents  device, [batch, latent_channels, latent_h, latent_w], NCHW, cfg.dtype
  *   frames   device, [batch, out_channels, 8*latent_h, 8*latent_w], NCHW, cfg.dtype; raw conv_out
- *            values (no clamp)
+ *            values (no clamp).  With VD_FLAG_OUT_U8: [batch, 8*latent_h, 8*latent_w, out_channels]
+ *            uint8 (see the flag)
  * Asynchronous on `cuda_stream`: enqueues kernels only, no allocation, no host synchronisation.
  * 1 <= batch <= cfg.max_batch.  Calls on one handle must not overlap (one workspace). */
 VD_API vd_status vd_decode(vd_handle h, const void* latents, void* frames, int32_t batch, void* cuda_stream);
@@ -123,6 +129,17 @@ VD_API vd_status vd_decode_extrapolated(vd_handle h, const void* z_prev, const v
  * part of the workspace. */
 VD_API vd_status vd_decode_host(vd_handle h, const void* latents_host, void* frames_host, int32_t batch,
                                 void* cuda_stream);
+
+/* A stream of frames through host memory with the copies hidden behind the decodes (Algorithm 1's loop:
+ * latents arrive, are decoded, frames are pushed to the output queue; Table II's "Data Transport" row, pinned
+ * memory).  latents_host holds n_frames latents, frames_host receives n_frames frames (layouts as in
+ * vd_decode, contiguous over frames).  Frames are decoded `batch` at a time (the last step may be smaller);
+ * while step t is decoded on `cuda_stream`, the latents of step t+1 travel to the device and the frames
+ * of step t-1 travel back, on two copy streams of the handle (created on the first call), through two
+ * staging buffers each in the workspace.  No host synchronisation per frame: the call returns once the
+ * last frame has reached the host.  Use pinned host memory: with pageable memory the copies do not overlap. */
+VD_API vd_status vd_decode_host_stream(vd_handle h, const void* latents_host, void* frames_host,
+                                       int32_t n_frames, int32_t batch, void* cuda_stream);
 
 /* Reads the device status word (call after the stream has been synchronised): VD_OK, or
  * VD_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait (every spin-wait inside the

@@ -44,7 +44,7 @@ typedef struct {
     int32_t has_residual;       /* 1: an fp32 residual tensor is added in the epilogue */
     int32_t phase_collapsed;    /* 1: an upsampling conv run as four 2x2 convolutions of the source (flops_per_frame
                                    still counts the layer's own 9 taps; the kernel executes 4/9 of them) */
-    int32_t reserved[1];
+    int32_t out_u8;             /* 1: the output is the display-packed uint8 NHWC frame (VD_FLAG_OUT_U8) */
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);

@@ -16,6 +16,7 @@ VD_F32, VD_BF16 = 0, 1
 VD_ARCH_TINY, VD_ARCH_SDVAE = 0, 1
 VD_FLAG_FORCE_SIMT = 0x1
 VD_FLAG_UPSAMPLE_9TAP = 0x2
+VD_FLAG_OUT_U8 = 0x4
 VD_IMPL_AUTO, VD_IMPL_SIMT, VD_IMPL_TC = 0, 1, 2
 VD_STEP_INGEST, VD_STEP_GN_STATS, VD_STEP_CONV, VD_STEP_ATTENTION = 0, 1, 2, 3
 STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", -3: "VD_ERR_WORKSPACE",
@@ -25,7 +26,7 @@ EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
     "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
-    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_debug_status_offset", "vd_debug_wait_probe",
+    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_decode_host_stream", "vd_debug_status_offset", "vd_debug_wait_probe",
 ]
 
 
@@ -45,7 +46,7 @@ class VdStepInfo(Structure):
                 ("out_h", c_int32), ("out_w", c_int32), ("out_channels", c_int32), ("out_dtype", c_int32),
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
                 ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
-                ("has_residual", c_int32), ("phase_collapsed", c_int32), ("reserved", c_int32 * 1)]
+                ("has_residual", c_int32), ("phase_collapsed", c_int32), ("out_u8", c_int32)]
 
 
 class VdConvDesc(Structure):
@@ -86,6 +87,7 @@ def lib():
         l.vd_profile.argtypes = [vp, vp, vp, c_int32, vp, POINTER(c_float), c_int32]
         l.vd_debug_stop_after.argtypes = [vp, c_int32]
         l.vd_clear_status.argtypes = [vp, vp]
+        l.vd_decode_host_stream.argtypes = [vp, vp, vp, c_int32, c_int32, vp]
         l.vd_debug_status_offset.argtypes = [vp, POINTER(c_int64)]
         l.vd_debug_wait_probe.argtypes = [vp, c_int64, vp]
         l.vd_conv_packed_weight_bytes.argtypes = [POINTER(VdConvDesc), POINTER(c_size_t)]
@@ -168,7 +170,10 @@ class Decoder:
         _check(lib().vd_create(byref(self.cfg), arr, len(dev_w), c_void_p(self.workspace.data_ptr()),
                                self.workspace_bytes, _stream_ptr(), byref(h)))
         self.handle = h
-        self.out_shape = (self.cfg.out_channels, 8 * latent_h, 8 * latent_w)
+        self.out_u8 = bool(flags & VD_FLAG_OUT_U8)
+        self.out_dtype = torch.uint8 if self.out_u8 else self.dtype
+        self.out_shape = ((8 * latent_h, 8 * latent_w, self.cfg.out_channels) if self.out_u8
+                          else (self.cfg.out_channels, 8 * latent_h, 8 * latent_w))
         self.latent_shape = (self.cfg.latent_channels, latent_h, latent_w)
 
     # ---- decode
@@ -179,7 +184,8 @@ class Decoder:
         b = latents.shape[0]
         assert tuple(latents.shape[1:]) == self.latent_shape
         if frames is None:
-            frames = torch.empty((b,) + self.out_shape, dtype=self.dtype, device=self.device)
+            frames = torch.empty((b,) + self.out_shape, dtype=self.out_dtype, device=self.device)
+        assert frames.dtype == self.out_dtype and frames.is_contiguous()
         _check(lib().vd_decode(self.handle, c_void_p(latents.data_ptr()), c_void_p(frames.data_ptr()), b,
                                _stream_ptr(stream)), self.handle)
         return frames
@@ -188,7 +194,7 @@ class Decoder:
         torch = self.torch
         b = z_prev.shape[0]
         if frames is None:
-            frames = torch.empty((b,) + self.out_shape, dtype=self.dtype, device=self.device)
+            frames = torch.empty((b,) + self.out_shape, dtype=self.out_dtype, device=self.device)
         z = torch.empty_like(z_prev) if want_state else None
         v = torch.empty_like(z_prev) if want_state else None
         _check(lib().vd_decode_extrapolated(
@@ -200,10 +206,22 @@ class Decoder:
     def decode_host(self, latents_host, frames_host, stream=None):
         """Host tensors in, host tensors out (pinned memory recommended); returns after the copy back."""
         assert not latents_host.is_cuda and not frames_host.is_cuda
-        assert latents_host.dtype == self.dtype and frames_host.dtype == self.dtype
+        assert latents_host.dtype == self.dtype and frames_host.dtype == self.out_dtype
         b = latents_host.shape[0]
         _check(lib().vd_decode_host(self.handle, c_void_p(latents_host.data_ptr()), c_void_p(frames_host.data_ptr()),
                                     b, _stream_ptr(stream)), self.handle)
+        return frames_host
+
+    def decode_host_stream(self, latents_host, frames_host, batch: int = 1, stream=None):
+        """A stream of frames through (pinned) host memory, `batch` per decode, copies overlapped with the
+        decodes; returns when the last frame has reached frames_host."""
+        assert not latents_host.is_cuda and not frames_host.is_cuda
+        assert latents_host.dtype == self.dtype and frames_host.dtype == self.out_dtype
+        assert latents_host.is_contiguous() and frames_host.is_contiguous()
+        n = latents_host.shape[0]
+        assert frames_host.shape[0] == n and tuple(frames_host.shape[1:]) == self.out_shape
+        _check(lib().vd_decode_host_stream(self.handle, c_void_p(latents_host.data_ptr()), c_void_p(frames_host.data_ptr()),
+                                           n, batch, _stream_ptr(stream)), self.handle)
         return frames_host
 
     # ---- introspection

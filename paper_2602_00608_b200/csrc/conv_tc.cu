@@ -672,7 +672,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             if (co < a.Cout) {
                                 const float v = __uint_as_float(r[co]) + (a.bias ? __ldg(a.bias + co) : 0.f);
                                 const size_t o = (((size_t)tl.b * a.Cout + co) * a.H + oy) * a.W + ox;
-                                if (a.out_dtype == VD_BF16) ((__nv_bfloat16*)a.y)[o] = __float2bfloat16_rn(v);
+                                if (a.out_u8) ((unsigned char*)a.y)[(((size_t)tl.b * a.H + oy) * a.W + ox) * a.Cout + co] = pack_u8(v);
+                                else if (a.out_dtype == VD_BF16) ((__nv_bfloat16*)a.y)[o] = __float2bfloat16_rn(v);
                                 else ((float*)a.y)[o] = v;
                             }
                         }
@@ -1396,8 +1397,8 @@ bool conv_tc_supported(const ConvArgs& a) {
     if (a.x2 && (a.Cin2 % 64 != 0 || a.Cin2 < 64)) return false;
     if (a.upsample == 2)     // phase-collapsed form: 3x3, 128-channel blocks, plain NHWC store
         return a.ksize == 3 && a.Cout % 128 == 0 && !a.out_nchw && !a.residual && !a.x2;
-    if (a.Cout % 128 == 0) return !a.out_nchw;
-    return a.Cout <= 16 && a.out_nchw && !a.residual && !a.x2;      // the frame head: Cout padded to 16
+    if (a.Cout % 128 == 0) return !a.out_nchw && !a.out_u8;
+    return a.Cout <= 16 && (a.out_nchw || a.out_u8) && !a.residual && !a.x2;      // the frame head: Cout padded to 16
 }
 
 bool conv_tc_pairs_available() { return pairs_available(); }
@@ -1478,7 +1479,7 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
     } else {
         memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
     }
-    if (!a.out_nchw) {
+    if (!a.out_nchw && !a.out_u8) {
         // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one epilogue warp's quarter (4 rows) of a 128-byte-wide slice of a tile
         const cuuint64_t dims[4] = {(cuuint64_t)a.Cout, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)std::max(a.B, 1)};
         const cuuint64_t strides[3] = {(cuuint64_t)a.Cout * es, (cuuint64_t)a.W * a.Cout * es, (cuuint64_t)a.H * a.W * a.Cout * es};
@@ -1500,7 +1501,7 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
 
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
     if (!plan.valid) return cudaErrorInvalidValue;
-    if (!a.out_nchw && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
+    if (!a.out_nchw && !a.out_u8 && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
     if ((a.upsample == 2) != (plan.phase != 0)) return cudaErrorInvalidValue;
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;

@@ -296,7 +296,8 @@ __global__ void __launch_bounds__((TH * TW / PPT) * CGROUPS) conv_simt_kernel(Co
             const size_t nhwc = (((size_t)b * a.H + oy) * a.W + ox) * a.Cout + co;
             if (a.residual) v += a.residual[nhwc];
             const size_t o = a.out_nchw ? (((size_t)b * a.Cout + co) * a.H + oy) * a.W + ox : nhwc;
-            st_f<TOut>(y, o, v);
+            if (a.out_u8) ((unsigned char*)a.y)[nhwc] = pack_u8(v);
+            else st_f<TOut>(y, o, v);
         }
     }
 }

@@ -50,8 +50,29 @@ struct vd_handle_s {
     std::vector<WeightJob> jobs;
     std::string err;
     int stop_after = -1;
-    size_t status_off = 0, lat_stage_off = 0, frm_stage_off = 0, gn_counter_off = 0;
+    size_t status_off = 0, lat_stage_off[2] = {0, 0}, frm_stage_off[2] = {0, 0}, gn_counter_off = 0;
     size_t total = 0;
+    // host-transport pipeline (vd_decode_host_stream): two copy streams and the events that order
+    // copies and decodes; created on first use, destroyed with the handle
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_dec[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    bool pipe_ready = false;
+    size_t frame_bytes(int batch) const {
+        const size_t px = (size_t)batch * cfg.out_channels * cfg.latent_h * cfg.latent_w * 64;
+        return (cfg.flags & VD_FLAG_OUT_U8) ? px : px * (cfg.dtype == VD_BF16 ? 2 : 4);
+    }
+    size_t latent_bytes(int batch) const {
+        return (size_t)batch * cfg.latent_channels * cfg.latent_h * cfg.latent_w * (cfg.dtype == VD_BF16 ? 2 : 4);
+    }
+    ~vd_handle_s() {
+        for (int i = 0; i < 2; ++i) {
+            if (ev_in[i]) cudaEventDestroy(ev_in[i]);
+            if (ev_dec[i]) cudaEventDestroy(ev_dec[i]);
+            if (ev_out[i]) cudaEventDestroy(ev_out[i]);
+        }
+        if (copy_in) cudaStreamDestroy(copy_in);
+        if (copy_out) cudaStreamDestroy(copy_out);
+    }
 };
 
 namespace {
@@ -118,7 +139,7 @@ class Planner {
     void add_conv(const std::string& name, const std::vector<std::string>& wnames, int Cout_each, size_t x_off,
                   int in_dtype, int Hs, int Ws, int Cin, int ksize, bool upsample, bool prologue, bool silu,
                   long residual_off, size_t y_off, int out_dtype, bool out_nchw, bool y_is_frames,
-                  const std::string& shortcut_name = std::string(), size_t x2_off = 0, int Cin2 = 0) {
+                  const std::string& shortcut_name = std::string(), size_t x2_off = 0, int Cin2 = 0, bool out_u8 = false) {
         Step s{};
         s.kind = VD_STEP_CONV;
         const int Cout = Cout_each * (int)wnames.size();
@@ -133,6 +154,7 @@ class Planner {
         a.Cin = Cin; a.Cout = Cout; a.ksize = ksize; a.upsample = upsample ? 1 : 0; a.silu = silu;
         a.in_dtype = in_dtype; a.out_dtype = out_dtype; a.out_nchw = out_nchw; a.bf16_operands = bf16();
         if (!shortcut_name.empty()) { a.x2 = ptr<void>(x2_off); a.Cin2 = Cin2; }
+        a.out_u8 = out_u8 ? 1 : 0;
         const bool tc_on = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT);
         ConvArgs probe = a;
         probe.B = 1;
@@ -159,7 +181,8 @@ class Planner {
         fill_info(s, name, tc, Cin, Cout, ksize, upsample, H, W, Cout, out_dtype, out_nchw, y_is_frames ? -1 : (long)y_off);
         const double P = (double)H * W;
         s.info.flops_per_frame = 2.0 * ksize * ksize * Cin * (double)Cout * P;
-        s.info.bytes_per_frame = (double)Hs * Ws * Cin * elt(in_dtype) + P * Cout * elt(out_dtype) +
+        s.info.out_u8 = out_u8 ? 1 : 0;
+        s.info.bytes_per_frame = (double)Hs * Ws * Cin * elt(in_dtype) + P * Cout * (out_u8 ? 1 : elt(out_dtype)) +
                                  (residual_off >= 0 ? P * Cout * 4.0 : 0.0);
         s.info.weight_bytes = (double)ksize * ksize * Cin * Cout * elt(cfg_.dtype);
         s.info.has_residual = residual_off >= 0;
@@ -285,8 +308,10 @@ class Planner {
         qkv_ = qkv ? alloc((size_t)B * qkv * ae) : 0;
         attno_ = ao ? alloc((size_t)B * ao * ae) : 0;
         vt_ = ao ? alloc(attn_tc_scratch_bytes(B, (int)P0, 512)) : 0;
-        h_->lat_stage_off = alloc((size_t)B * P0 * lc * elt(cfg_.dtype));
-        h_->frm_stage_off = alloc((size_t)B * P0 * 64 * cfg_.out_channels * elt(cfg_.dtype));
+        for (int i = 0; i < 2; ++i) {        // two of each: a copy runs while the other buffer is decoded from / into
+            h_->lat_stage_off[i] = alloc((size_t)B * P0 * lc * elt(cfg_.dtype));
+            h_->frm_stage_off[i] = alloc((size_t)B * P0 * 64 * cfg_.out_channels * elt(cfg_.dtype));
+        }
 
         // ---- steps
         {
@@ -341,8 +366,9 @@ class Planner {
 
     void head(int C, int H, int W) {
         add_gn("norm_out", xs_[cur_x_], VD_F32, H, W, C, "norm_out");
+        const bool u8 = (cfg_.flags & VD_FLAG_OUT_U8) != 0;
         add_conv("conv_out", {"conv_out"}, cfg_.out_channels, xs_[cur_x_], VD_F32, H, W, C, 3, false, true, true, -1, 0,
-                 cfg_.dtype, true, true);
+                 cfg_.dtype, !u8, true, std::string(), 0, 0, u8);
     }
 
   private:
@@ -371,7 +397,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP | VD_FLAG_OUT_U8)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -436,7 +462,8 @@ vd_status decode_impl(vd_handle h, const void* latents, const void* v_prev, floa
     if (!latents || !frames) return fail(h, VD_ERR_INVALID_ARG, "latents/frames must not be NULL");
     if (batch < 1 || batch > h->cfg.max_batch) return fail(h, VD_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
     const size_t al = h->cfg.dtype == VD_BF16 ? 2 : 4;
-    if (((uintptr_t)latents % al) || ((uintptr_t)frames % al)) return fail(h, VD_ERR_INVALID_ARG, "latents/frames are misaligned for their dtype");
+    const size_t fal = (h->cfg.flags & VD_FLAG_OUT_U8) ? 1 : al;
+    if (((uintptr_t)latents % al) || ((uintptr_t)frames % fal)) return fail(h, VD_ERR_INVALID_ARG, "latents/frames are misaligned for their dtype");
     cudaStream_t s = (cudaStream_t)stream;
     const int n = h->stop_after >= 0 ? std::min((int)h->steps.size(), h->stop_after + 1) : (int)h->steps.size();
     std::vector<cudaEvent_t> ev;
@@ -578,11 +605,9 @@ vd_status vd_decode_host(vd_handle h, const void* latents_host, void* frames_hos
     if (!latents_host || !frames_host) return fail(h, VD_ERR_INVALID_ARG, "host buffers must not be NULL");
     if (batch < 1 || batch > h->cfg.max_batch) return fail(h, VD_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
     cudaStream_t s = (cudaStream_t)cuda_stream;
-    const size_t es = elt(h->cfg.dtype);
-    const size_t lat_bytes = (size_t)batch * h->cfg.latent_channels * h->cfg.latent_h * h->cfg.latent_w * es;
-    const size_t frm_bytes = (size_t)batch * h->cfg.out_channels * h->cfg.latent_h * h->cfg.latent_w * 64 * es;
-    void* dl = h->ws + h->lat_stage_off;
-    void* df = h->ws + h->frm_stage_off;
+    const size_t lat_bytes = h->latent_bytes(batch), frm_bytes = h->frame_bytes(batch);
+    void* dl = h->ws + h->lat_stage_off[0];
+    void* df = h->ws + h->frm_stage_off[0];
     cudaError_t e = cudaMemcpyAsync(dl, latents_host, lat_bytes, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail(h, e, "latents host-to-device copy");
     vd_status st = decode_impl(h, dl, nullptr, 0.f, nullptr, nullptr, df, batch, cuda_stream, nullptr, 0);
@@ -592,6 +617,68 @@ vd_status vd_decode_host(vd_handle h, const void* latents_host, void* frames_hos
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(h, e, "vd_decode_host synchronise");
     return VD_OK;
+}
+
+vd_status vd_decode_host_stream(vd_handle h, const void* latents_host, void* frames_host, int32_t n_frames,
+                                int32_t batch, void* cuda_stream) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (!latents_host || !frames_host) return fail(h, VD_ERR_INVALID_ARG, "host buffers must not be NULL");
+    if (batch < 1 || batch > h->cfg.max_batch) return fail(h, VD_ERR_INVALID_ARG, "batch must be in [1, max_batch]");
+    if (n_frames < 0) return fail(h, VD_ERR_INVALID_ARG, "n_frames must not be negative");
+    if (n_frames == 0) return VD_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaSuccess;
+    if (!h->pipe_ready) {
+        e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_dec[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_out[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return cuda_fail(h, e, "vd_decode_host_stream set-up");
+        h->pipe_ready = true;
+    }
+    const int steps = (n_frames + batch - 1) / batch;
+    const size_t lat1 = h->latent_bytes(1), frm1 = h->frame_bytes(1);
+    auto frames_of = [&](int t) { return std::min(batch, n_frames - t * batch); };
+    // Work of earlier calls on `cuda_stream` (and whatever it waits for) comes first: the copy streams join it.
+    e = cudaEventRecord(h->ev_dec[0], s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_in, h->ev_dec[0], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_dec[0], 0);
+    auto copy_in = [&](int t) -> cudaError_t {        // latents of step t -> device buffer t & 1
+        const int k = t & 1;
+        cudaError_t ce = cudaSuccess;
+        if (t >= 2) ce = cudaStreamWaitEvent(h->copy_in, h->ev_dec[k], 0);          // the decode that read this buffer is done
+        if (ce == cudaSuccess)
+            ce = cudaMemcpyAsync(h->ws + h->lat_stage_off[k], (const char*)latents_host + (size_t)t * batch * lat1,
+                                 lat1 * frames_of(t), cudaMemcpyHostToDevice, h->copy_in);
+        if (ce == cudaSuccess) ce = cudaEventRecord(h->ev_in[k], h->copy_in);
+        return ce;
+    };
+    if (e == cudaSuccess) e = copy_in(0);
+    for (int t = 0; t < steps && e == cudaSuccess; ++t) {
+        const int k = t & 1;
+        if (t + 1 < steps) e = copy_in(t + 1);                                       // next latents travel during this decode
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, h->ev_in[k], 0);
+        if (e == cudaSuccess && t >= 2) e = cudaStreamWaitEvent(s, h->ev_out[k], 0); // the copy that read this frame buffer is done
+        if (e != cudaSuccess) break;
+        vd_status st = decode_impl(h, h->ws + h->lat_stage_off[k], nullptr, 0.f, nullptr, nullptr, h->ws + h->frm_stage_off[k],
+                                   frames_of(t), cuda_stream, nullptr, 0);
+        if (st != VD_OK) { cudaStreamSynchronize(h->copy_in); cudaStreamSynchronize(h->copy_out); cudaStreamSynchronize(s); return st; }
+        e = cudaEventRecord(h->ev_dec[k], s);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_dec[k], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync((char*)frames_host + (size_t)t * batch * frm1, h->ws + h->frm_stage_off[k], frm1 * frames_of(t),
+                                cudaMemcpyDeviceToHost, h->copy_out);                // previous frames travel during the next decode
+        if (e == cudaSuccess) e = cudaEventRecord(h->ev_out[k], h->copy_out);
+    }
+    // one wait at the end: every frame has reached the host, and `cuda_stream` is idle again
+    cudaError_t e2 = cudaStreamSynchronize(h->copy_out);
+    cudaError_t e3 = cudaStreamSynchronize(s);
+    cudaError_t e4 = cudaStreamSynchronize(h->copy_in);
+    if (e == cudaSuccess) e = e2 != cudaSuccess ? e2 : (e3 != cudaSuccess ? e3 : e4);
+    return e == cudaSuccess ? VD_OK : cuda_fail(h, e, "vd_decode_host_stream");
 }
 
 vd_status vd_get_status(vd_handle h) {

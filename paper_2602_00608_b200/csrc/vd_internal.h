@@ -26,6 +26,7 @@ struct ConvArgs {
                             // (four 2x2 convolutions of the source with pre-summed weights; tensor-core kernel only)
     int silu;
     int in_dtype, out_dtype, out_nchw, bf16_operands;
+    int out_u8;             // 1: y is the display-packed frame, NHWC uint8 [B,H,W,Cout] (out_dtype and out_nchw are ignored)
     // optional fused 1x1 shortcut (tensor-core kernel only): y += W2 * x2 + bias2
     const void* x2;         // fp32 NHWC [B,H,W,Cin2] at the output resolution, or null
     const void* w2;         // packed bf16 [Cout][Cin2]
@@ -151,6 +152,14 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 }
 
 #ifdef __CUDACC__
+// Display packing of one frame value for transport: [-1, 1] -> 0..255, t = fma(x, 127.5, 127.5) in fp32 (one
+// rounding), clamped, rounded to nearest with ties to even; NaN packs to 0.
+__device__ __forceinline__ unsigned char pack_u8(float x) {
+    float t = fmaf(x, 127.5f, 127.5f);
+    t = t > 0.f ? t : 0.f;
+    t = fminf(t, 255.f);
+    return (unsigned char)__float2int_rn(t);
+}
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
