@@ -54,6 +54,9 @@ WORKLOADS = {
     3: Workload(3, "sdvae-bf16-720x480", ARCH_SDVAE, "bf16", 1, 60, 90, 32, 1e-6, 1002, 2003, "normal_scaled"),
     4: Workload(4, "sdvae-bf16-720x480-stream8", ARCH_SDVAE, "bf16", 8, 60, 90, 32, 1e-6, 1002, 2004, "ar1"),
     5: Workload(5, "sdvae-bf16-1280x720-b2", ARCH_SDVAE, "bf16", 2, 90, 160, 32, 1e-6, 1002, 2005, "normal"),
+    # beyond the benchmark's list: the paper's second workload shape, the 256x256 platformer frames (Section V,
+    # experimental setup; Table III, first row), as a stream of four AR(1) latents of 32x32
+    6: Workload(6, "sdvae-bf16-256x256-stream4", ARCH_SDVAE, "bf16", 4, 32, 32, 32, 1e-6, 1002, 2006, "ar1"),
 }
 
 SDVAE_LEVEL_CHANNELS = (512, 512, 256, 128)

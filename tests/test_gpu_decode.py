@@ -149,6 +149,22 @@ def test_full_size_configs_whole_frame_against_the_oracle(env, idx):
     assert r2 <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
 
 
+def test_platformer_shape_256x256_stream_against_the_oracle(env):
+    """The paper's second workload shape (256x256 frames, latent 32x32), four AR(1) frames in one batch:
+    every pixel of the first and last frame against the oracle run in the test."""
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[6]
+    z = synth.workload_latents(wl)
+    dec, got, wts = _decode(env, wl, z)
+    assert got.shape == (4, 3, 256, 256)
+    for b in (0, 3):
+        want = ref.decode(wl.arch, wts, z[b:b + 1], wl.groups, wl.eps)[0]
+        g = got[b].float().cpu().numpy()
+        r, m = rel_l2(g, want), max_abs(g, want)
+        print(f"whole-frame parity {wl.name} frame {b}: rel-L2 {r:.3e} max-abs {m:.3e}")
+        assert r <= BF16_REL_L2 and m <= BF16_MAX_ABS, (b, r, m)
+
+
 def test_host_buffer_decode_and_extrapolation(env):
     torch, ref, vd, synth = env
     wl = synth.WORKLOADS[2]
