@@ -1,7 +1,7 @@
 """Micro-benchmark of one fused convolution layer through the C ABI (vd_op_conv2d), for profiling a
 single kernel on a small case.
 
-    python -m paper_2602_00608_b200.bench_layer --h 240 --w 360 --cin 256 --cout 256 [--in-f32]
+    python bench_layer.py --h 240 --w 360 --cin 256 --cout 256 [--in-f32]
         [--out-f32] [--residual] [--prologue] [--upsample] [--k 3] [--iters 5] [--batch 1]
 
 Prints one JSON line with the mean device time (CUDA events on the launching stream) and the
@@ -15,7 +15,11 @@ import json
 
 import torch
 
-from . import binding as vd
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+from paper_2602_00608_b200 import binding as vd  # noqa: E402
 
 
 def main():

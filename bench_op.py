@@ -1,8 +1,8 @@
 """Micro-benchmark of the two other operators of the decoder through the C ABI, for profiling a single
 kernel on a small case:
 
-    python -m paper_2602_00608_b200.bench_op gn --h 480 --w 720 --c 128 [--f32] [--iters 5]
-    python -m paper_2602_00608_b200.bench_op attn --tokens 5400 --c 512 [--iters 5]
+    python bench_op.py gn --h 480 --w 720 --c 128 [--f32] [--iters 5]
+    python bench_op.py attn --tokens 5400 --c 512 [--iters 5]
 
 gn:   GroupNorm statistics (vd_op_gn_stats) of an NHWC tensor, 32 groups; prints the mean device time and the
       achieved GB/s (algorithmic bytes: one read of the tensor).
@@ -17,7 +17,11 @@ import json
 
 import torch
 
-from . import binding as vd
+import os
+import sys
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+from paper_2602_00608_b200 import binding as vd  # noqa: E402
 
 
 def _time(fn, iters, warmup):

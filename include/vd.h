@@ -59,6 +59,8 @@ typedef enum { VD_ARCH_TINY = 0, VD_ARCH_SDVAE = 1 } vd_arch;
                                      uint8 [batch, 8*latent_h, 8*latent_w, out_channels], q = round(clamp(x*0.5+0.5,
                                      0, 1)*255), computed in fp32 as rint(clamp(fma(x, 127.5, 127.5), 0, 255)) with ties
                                      to even, in the last convolution's epilogue (a quarter / half of the bytes to copy) */
+#define VD_FLAG_CANARY 0x8u       /* debugging: every workspace region is followed by a 256-byte guard pattern that
+                                     vd_debug_check_canaries (vd_ops.h) verifies; costs a little workspace, no time */
 #define VD_FLAG_UPSAMPLE_9TAP 0x2u /* upsampling convolutions as 9 taps on the 2x grid (upsampling folded into the
                                      addressing) instead of the default phase-collapsed form: per output parity a
                                      2x2 convolution of the source with pre-summed weights, 4/9 of the products,

@@ -67,6 +67,11 @@ VD_API vd_status vd_profile(vd_handle h, const void* latents, void* frames, int3
 VD_API vd_status vd_debug_status_offset(vd_handle h, int64_t* offset);
 VD_API vd_status vd_debug_wait_probe(vd_handle h, int64_t limit_cycles, void* cuda_stream);
 
+/* Debug (handles created with VD_FLAG_CANARY): synchronises the device and verifies the guard pattern behind
+ * every workspace region; VD_ERR_WORKSPACE (with the guard's index and offset in vd_last_error) if a kernel
+ * wrote outside its buffer.  *n_guards (may be NULL) receives the number of guards (0 without the flag). */
+VD_API vd_status vd_debug_check_canaries(vd_handle h, int32_t* n_guards);
+
 /* Debug: makes vd_decode stop after step `index` (so that step's output can be read from the
  * workspace at out_offset); -1 restores the full decode. */
 VD_API vd_status vd_debug_stop_after(vd_handle h, int32_t index);

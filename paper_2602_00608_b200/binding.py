@@ -17,6 +17,7 @@ VD_ARCH_TINY, VD_ARCH_SDVAE = 0, 1
 VD_FLAG_FORCE_SIMT = 0x1
 VD_FLAG_UPSAMPLE_9TAP = 0x2
 VD_FLAG_OUT_U8 = 0x4
+VD_FLAG_CANARY = 0x8
 VD_IMPL_AUTO, VD_IMPL_SIMT, VD_IMPL_TC = 0, 1, 2
 VD_STEP_INGEST, VD_STEP_GN_STATS, VD_STEP_CONV, VD_STEP_ATTENTION = 0, 1, 2, 3
 STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", -3: "VD_ERR_WORKSPACE",
@@ -26,7 +27,7 @@ EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
     "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
-    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_decode_host_stream", "vd_debug_status_offset", "vd_debug_wait_probe",
+    "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_decode_host_stream", "vd_debug_check_canaries", "vd_debug_status_offset", "vd_debug_wait_probe",
 ]
 
 
@@ -88,6 +89,7 @@ def lib():
         l.vd_debug_stop_after.argtypes = [vp, c_int32]
         l.vd_clear_status.argtypes = [vp, vp]
         l.vd_decode_host_stream.argtypes = [vp, vp, vp, c_int32, c_int32, vp]
+        l.vd_debug_check_canaries.argtypes = [vp, POINTER(c_int32)]
         l.vd_debug_status_offset.argtypes = [vp, POINTER(c_int64)]
         l.vd_debug_wait_probe.argtypes = [vp, c_int64, vp]
         l.vd_conv_packed_weight_bytes.argtypes = [POINTER(VdConvDesc), POINTER(c_size_t)]
@@ -239,6 +241,12 @@ class Decoder:
 
     def wait_probe(self, limit_cycles: int, stream=None):
         _check(lib().vd_debug_wait_probe(self.handle, limit_cycles, _stream_ptr(stream)), self.handle)
+
+    def check_canaries(self) -> int:
+        """Verifies the workspace guards (handles created with VD_FLAG_CANARY); returns their number."""
+        n = c_int32(0)
+        _check(lib().vd_debug_check_canaries(self.handle, byref(n)), self.handle)
+        return int(n.value)
 
     def steps(self):
         n = c_int32(0)

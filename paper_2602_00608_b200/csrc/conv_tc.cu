@@ -89,13 +89,13 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // chunk therefore stays in shared memory for four slots (five stages).  PhaseSched is that schedule; the
 // weight loader follows it step by step.
 template <int BN, int CG = 1, bool PH = false> struct TileCfg {
-    static_assert(CG == 1 || BN == 256 || PH, "the two-CTA form exists for 256-channel blocks and the phase form");
+    static_assert(CG == 1 || BN >= 128, "the two-CTA form exists for 128- and 256-channel blocks");
     static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
     static constexpr int PAIR = PH ? 1 : (BN == 256 ? 1 : 2);        // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (PH ? 2 : 1) * (BN / CG) * 128;   // this CTA's rows x 64 bf16 (phase: two taps)
     static constexpr int OUT_BUFS = PH ? 2 : 1;                      // output slices per epilogue warp
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
-    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? 7 : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
+    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = PH ? 5 : 2;                    // phase form: a chunk stays until the parity that lags most has used it
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
@@ -148,13 +148,17 @@ struct Sched {
         r.tx0 = (s - row * tiles_x) * TILE_W;
         return r;
     }
-    // number of tiles of the item that starts at tile t
+    // number of tiles of the item that starts at tile t: up to pair * cg consecutive tiles of one (frame, channel block)
     __device__ __forceinline__ int count(int t) const {
-        return ((pair == 2 || cg == 2) && t + 1 < end && fdiv(t + 1, m_tiles) == fdiv(t, m_tiles)) ? 2 : 1;
+        const int cap = pair * cg;
+        const int blk = fdiv(t, m_tiles);
+        int n = 1;
+        while (n < cap && t + n < end && fdiv(t + n, m_tiles) == blk) ++n;
+        return n;
     }
-    // of those, the tiles this CTA works on, and the s-th of them
-    __device__ __forceinline__ int mine(int n) const { return cg == 2 ? (rank < n ? 1 : 0) : n; }
-    __device__ __forceinline__ int index(int t, int s) const { return cg == 2 ? t + rank : t + s; }
+    // of those, the tiles this CTA works on (the pair's CTAs take alternate tiles), and the s-th of them
+    __device__ __forceinline__ int mine(int n) const { return cg == 2 ? ((n - rank + 1) >> 1) : n; }
+    __device__ __forceinline__ int index(int t, int s) const { return cg == 2 ? t + 2 * s + rank : t + s; }
 };
 
 // The phase form's order of (parity, chunk) blocks.  The CTA's work is a sequence of chunk slots
@@ -354,17 +358,23 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 p.tile = sched.get(p.cnt > 0 ? sched.index(p.t, 0) : p.t, BN);
             };
             auto advance = [&](Pos& p) {
-                if (++p.slot < p.cnt) {                          // the item's second tile: the next one of its channel block
-                    p.tile.tx0 += TILE_W;
-                    if (p.tile.tx0 >= sched.tiles_x * TILE_W) { p.tile.tx0 = 0; p.tile.ty0 += TILE_H; }
+                if (++p.slot < p.cnt) {                          // the item's second tile of this CTA: CG tiles on in its channel block
+#pragma unroll
+                    for (int k = 0; k < CG; ++k) {
+                        p.tile.tx0 += TILE_W;
+                        if (p.tile.tx0 >= sched.tiles_x * TILE_W) { p.tile.tx0 = 0; p.tile.ty0 += TILE_H; }
+                    }
                     return;
                 }
                 const bool two = p.slot == 2;
                 p.slot = 0;
                 if (++p.kc < ktotal) {                           // next chunk of the same item: back to its first tile
                     if (two) {
-                        if (p.tile.tx0 == 0) { p.tile.tx0 = (sched.tiles_x - 1) * TILE_W; p.tile.ty0 -= TILE_H; }
-                        else p.tile.tx0 -= TILE_W;
+#pragma unroll
+                        for (int k = 0; k < CG; ++k) {
+                            if (p.tile.tx0 == 0) { p.tile.tx0 = (sched.tiles_x - 1) * TILE_W; p.tile.ty0 -= TILE_H; }
+                            else p.tile.tx0 -= TILE_W;
+                        }
                     }
                     return;
                 }

@@ -38,6 +38,8 @@ struct WeightJob {           // repack work done once in vd_create
 };
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardByte = 0xA5;
 int elt(int dtype) { return dtype == VD_BF16 ? 2 : 4; }
 
 }  // namespace
@@ -48,6 +50,7 @@ struct vd_handle_s {
     size_t ws_bytes = 0;
     std::vector<Step> steps;
     std::vector<WeightJob> jobs;
+    std::vector<size_t> guards;          // offsets of the guard regions (VD_FLAG_CANARY)
     std::string err;
     int stop_after = -1;
     size_t status_off = 0, lat_stage_off[2] = {0, 0}, frm_stage_off[2] = {0, 0}, gn_counter_off = 0;
@@ -83,9 +86,17 @@ class Planner {
   public:
     Planner(vd_handle_s* h, char* base) : h_(h), base_(base), cfg_(h->cfg) {}
 
+    // With VD_FLAG_CANARY every region is followed by a 256-byte guard that vd_create fills with a pattern
+    // and vd_debug_check_canaries verifies: a kernel that writes past the end of its buffer (or before the start of
+    // the next one) is caught even if the overrun lands in memory that a later layer overwrites.
     size_t alloc(size_t bytes) {
         const size_t off = align_up(cur_, 256);
         cur_ = off + bytes;
+        if (cfg_.flags & VD_FLAG_CANARY) {
+            const size_t g = align_up(cur_, 256);
+            h_->guards.push_back(g);
+            cur_ = g + kGuardBytes;
+        }
         return off;
     }
     template <typename T> T* ptr(size_t off) const { return (T*)(base_ + off); }
@@ -397,7 +408,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP | VD_FLAG_OUT_U8)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP | VD_FLAG_OUT_U8 | VD_FLAG_CANARY)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -549,6 +560,8 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
     e = cudaMemsetAsync(h->ws + h->status_off, 0, 256, s);
     // arrival counters of the GroupNorm statistics kernel: zero once, every launch leaves them zero
     if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + h->gn_counter_off, 0, (size_t)cfg->max_batch * 4, s);
+    for (size_t g : h->guards)
+        if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + g, kGuardByte, kGuardBytes, s);
     if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "status memset"); }
     for (const WeightJob& j : h->jobs) {
         const vd_tensor* t = find_tensor(weights, n_weights, j.name);
@@ -741,6 +754,27 @@ vd_status vd_debug_wait_probe(vd_handle h, int64_t limit_cycles, void* cuda_stre
         return fail(h, VD_ERR_INVALID_ARG, "limit_cycles must be in [1e3, 2e9]");
     cudaError_t e = launch_wait_probe((unsigned int*)(h->ws + h->status_off), (long long)limit_cycles, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? VD_OK : cuda_fail(h, e, "vd_debug_wait_probe");
+}
+
+vd_status vd_debug_check_canaries(vd_handle h, int32_t* n_guards) {
+    if (!h) return fail(nullptr, VD_ERR_INVALID_ARG, "handle is NULL");
+    if (n_guards) *n_guards = (int32_t)h->guards.size();
+    if (h->guards.empty()) return VD_OK;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(h, e, "vd_debug_check_canaries synchronise");
+    std::vector<unsigned char> host(kGuardBytes);
+    for (size_t i = 0; i < h->guards.size(); ++i) {
+        e = cudaMemcpy(host.data(), h->ws + h->guards[i], kGuardBytes, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(h, e, "vd_debug_check_canaries copy");
+        for (size_t k = 0; k < kGuardBytes; ++k)
+            if (host[k] != (unsigned char)kGuardByte) {
+                char msg[160];
+                snprintf(msg, sizeof(msg), "workspace guard %zu (offset %zu) was overwritten at byte %zu: a kernel wrote outside its buffer",
+                         i, h->guards[i], k);
+                return fail(h, VD_ERR_WORKSPACE, msg);
+            }
+    }
+    return VD_OK;
 }
 
 vd_status vd_debug_stop_after(vd_handle h, int32_t index) {

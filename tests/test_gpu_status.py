@@ -70,3 +70,29 @@ def test_clear_and_probe_reject_null_handles(dec_env):
     assert vd.lib().vd_clear_status(None, None) == vd.VD_ERR_INVALID_ARG
     assert vd.lib().vd_debug_wait_probe(None, 100000, None) == vd.VD_ERR_INVALID_ARG
     assert vd.lib().vd_debug_status_offset(dec.handle, None) == vd.VD_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("idx,flags", [(1, 0), (2, 0), (2, 1), (2, 4)])
+def test_workspace_guards_survive_decodes_and_catch_a_planted_overrun(idx, flags):
+    """Every workspace region of a handle created with VD_FLAG_CANARY is followed by a guard pattern: odd-sized,
+    batched decodes on every kernel path leave all guards intact, and a byte planted from the host is reported."""
+    import torch
+    from paper_2602_00608_b200 import binding as vd, synth
+    wl = synth.WORKLOADS[idx]
+    wts = synth.workload_weights(wl)
+    h, w, b = 11, 13, 3
+    dec = vd.Decoder(wl.arch, wl.dtype, h, w, b, wl.groups, wl.eps, wts, flags | vd.VD_FLAG_CANARY)
+    plain = vd.Decoder(wl.arch, wl.dtype, h, w, b, wl.groups, wl.eps, wts, flags)
+    z = torch.from_numpy(synth.workload_latents(wl, batch=b, h=h, w=w)).to("cuda:0", dec.dtype)
+    got = dec.decode(z)
+    dec.decode(z[:2].contiguous())
+    n = dec.check_canaries()
+    assert n > 50
+    assert torch.equal(got, plain.decode(z))                 # the guards change the layout, not the result
+    assert plain.check_canaries() == 0
+    # plant an overrun: the workspace ends with the guard of its last region; overwrite that guard's last byte
+    off = int(vd.query_workspace(dec.cfg))
+    dec.workspace[off - 1] = 0
+    with pytest.raises(vd.VdError) as e:
+        dec.check_canaries()
+    assert e.value.status == vd.VD_ERR_WORKSPACE and "guard" in str(e.value)
