@@ -10,6 +10,7 @@
 // S is double-buffered in TMEM (2 x 128 columns next to the 256 columns of O), so the tensor
 // core works on the next tile's scores while the softmax warps are busy.  The N x N score
 // matrix never exists in memory.  Every wait is bounded (see tc_common.cuh).
+#include <mutex>
 #include <cuda.h>
 
 #include "tc_common.cuh"
@@ -357,7 +358,22 @@ bool attn_tc_supported(const AttnArgs& a) {
 
 size_t attn_tc_scratch_bytes(int B, int T, int C) { return (size_t)B * C * padded_tokens(T) * 2; }
 
-cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status, cudaStream_t s) {
+cudaError_t attn_tc_prepare(const AttnArgs& a, AttnTcPlan* plan) {
+    plan->valid = 0;
+    if (!a.vt) return cudaErrorInvalidValue;
+    if (((uintptr_t)a.q | (uintptr_t)a.k | (uintptr_t)a.vt) & 15) return cudaErrorMisalignedAddress;
+    const int Tp = padded_tokens(a.T);
+    const uint64_t rows = (uint64_t)a.B * a.T;
+    if (!encode_2d((CUtensorMap*)plan->tq, a.q, a.C, rows, (uint64_t)a.ld_qkv * 2, DCHUNK, BQ)) return cudaErrorInvalidValue;
+    if (!encode_2d((CUtensorMap*)plan->tk, a.k, a.C, rows, (uint64_t)a.ld_qkv * 2, DCHUNK, BKV)) return cudaErrorInvalidValue;
+    if (!encode_2d((CUtensorMap*)plan->tv, a.vt, Tp, (uint64_t)a.B * a.C, (uint64_t)Tp * 2, 64, DV)) return cudaErrorInvalidValue;
+    plan->q = a.q; plan->k = a.k; plan->vt = a.vt;
+    plan->batch = a.B; plan->tokens = a.T;
+    plan->valid = 1;
+    return cudaSuccess;
+}
+
+cudaError_t launch_attn_tc(const AttnArgs& a, const AttnTcPlan* plan, unsigned int* status, cudaStream_t s) {
     if (!a.vt) return cudaErrorInvalidValue;
     if (((uintptr_t)a.q | (uintptr_t)a.k | (uintptr_t)a.v | (uintptr_t)a.o | (uintptr_t)a.vt) & 15) return cudaErrorMisalignedAddress;
     const int Tp = padded_tokens(a.T);
@@ -366,16 +382,28 @@ cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status, cudaStream_t
         cudaError_t e = launch_pdl(transpose_v_kernel, grid, block, 0, s, (const __nv_bfloat16*)a.v, (__nv_bfloat16*)a.vt, a.T, Tp, a.C, a.ld_qkv);
         if (e != cudaSuccess) return e;
     }
-    CUtensorMap tq, tk, tv;
-    const uint64_t rows = (uint64_t)a.B * a.T;
-    if (!encode_2d(&tq, a.q, a.C, rows, (uint64_t)a.ld_qkv * 2, DCHUNK, BQ)) return cudaErrorInvalidValue;
-    if (!encode_2d(&tk, a.k, a.C, rows, (uint64_t)a.ld_qkv * 2, DCHUNK, BKV)) return cudaErrorInvalidValue;
-    if (!encode_2d(&tv, a.vt, Tp, (uint64_t)a.B * a.C, (uint64_t)Tp * 2, 64, DV)) return cudaErrorInvalidValue;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL);
+    // The maps of a decoder's fixed workspace tensors are built once (attn_tc_prepare, for the largest batch: rows
+    // beyond the batch in use are never addressed); a call on other tensors encodes its own.
+    AttnTcPlan local;
+    if (!(plan && plan->valid && plan->q == a.q && plan->k == a.k && plan->vt == a.vt && plan->tokens == a.T && a.B <= plan->batch)) {
+        cudaError_t e = attn_tc_prepare(a, &local);
         if (e != cudaSuccess) return e;
-        configured = true;
+        plan = &local;
+    }
+    const CUtensorMap &tq = *(const CUtensorMap*)plan->tq, &tk = *(const CUtensorMap*)plan->tk, &tv = *(const CUtensorMap*)plan->tv;
+    {
+        static std::mutex mu;
+        static bool configured[64] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {              // the attribute is per device
+            e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL);
+            if (e != cudaSuccess) return e;
+            configured[dev] = true;
+        }
     }
     AttnTcParams p{a.o, a.B, a.T, a.C, a.ld_o, a.scale * 1.4426950408889634f};
     dim3 grid((a.T + BQ - 1) / BQ, a.C / DV, a.B);

@@ -93,9 +93,9 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
     static constexpr int PAIR = PH ? 1 : (BN == 256 ? 1 : 2);        // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (PH ? 2 : 1) * (BN / CG) * 128;   // this CTA's rows x 64 bf16 (phase: two taps)
-    static constexpr int OUT_BUFS = PH ? 2 : 1;                      // output slices per epilogue warp
+    static constexpr int OUT_BUFS = (PH || BN == 128) ? 2 : 1;   // 128-channel blocks: a second slice buffer pays more than a fourth weight stage                      // output slices per epilogue warp
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
-    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? 4 : 8)));
+    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? 3 : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = PH ? 5 : 2;                    // phase form: a chunk stays until the parity that lags most has used it
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;

@@ -23,6 +23,7 @@ struct Step {
     AttnArgs attn;
     IngestArgs ing;
     ConvTcPlan tc;
+    AttnTcPlan attn_tc;
     // batch-dependent pointers are rebased per call: strides per frame
     bool has_residual;
 };
@@ -450,7 +451,7 @@ cudaError_t launch_step(const vd_handle_s* h, const Step& st, int B, const void*
         case VD_STEP_ATTENTION: {
             AttnArgs a = st.attn;
             a.B = B;
-            return st.use_tc ? launch_attn_tc(a, status, s) : launch_attn_simt(a, s);
+            return st.use_tc ? launch_attn_tc(a, &st.attn_tc, status, s) : launch_attn_simt(a, s);
         }
     }
     return cudaErrorInvalidValue;
@@ -595,6 +596,14 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
                                                          "upsampling convolution; set VD_FLAG_UPSAMPLE_9TAP");
             }
             if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "weight tensor map"); }
+        }
+    }
+    for (Step& st : h->steps) {
+        if (st.kind == VD_STEP_ATTENTION && st.use_tc) {
+            AttnArgs pa = st.attn;
+            pa.B = cfg->max_batch;
+            e = attn_tc_prepare(pa, &st.attn_tc);
+            if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "attention tensor maps"); }
         }
     }
     e = cudaStreamSynchronize(s);
@@ -914,7 +923,7 @@ vd_status vd_op_attention(const void* q, const void* k, const void* v, void* o, 
     const bool can = attn_tc_supported(a) && scratch != nullptr;
     if (impl == VD_IMPL_TC && !can) return fail(nullptr, VD_ERR_UNSUPPORTED, "the tensor-core attention does not support this shape");
     const bool tc = impl == VD_IMPL_TC || (impl == VD_IMPL_AUTO && can);
-    cudaError_t e = tc ? launch_attn_tc(a, nullptr, (cudaStream_t)cuda_stream) : launch_attn_simt(a, (cudaStream_t)cuda_stream);
+    cudaError_t e = tc ? launch_attn_tc(a, nullptr, nullptr, (cudaStream_t)cuda_stream) : launch_attn_simt(a, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_attention");
 }
 

@@ -116,7 +116,14 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan);      // a.w mu
 cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status_word, cudaStream_t s);
 bool attn_tc_supported(const AttnArgs& a);
 size_t attn_tc_scratch_bytes(int B, int T, int C);
-cudaError_t launch_attn_tc(const AttnArgs& a, unsigned int* status_word, cudaStream_t s);
+// Launch-invariant state of the tensor-core attention: the TMA descriptors of q, k and the transposed v.
+struct alignas(64) AttnTcPlan {
+    unsigned char tq[128], tk[128], tv[128];
+    const void* q; const void* k; const void* vt;
+    int batch, tokens, valid;
+};
+cudaError_t attn_tc_prepare(const AttnArgs& a, AttnTcPlan* plan);      // a.B = the largest batch the plan must serve
+cudaError_t launch_attn_tc(const AttnArgs& a, const AttnTcPlan* plan, unsigned int* status_word, cudaStream_t s);
 
 
 // ---- programmatic dependent launch
