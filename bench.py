@@ -203,6 +203,9 @@ def main():
     ap.add_argument("--impl", default="vd", choices=["vd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="force the FFMA cross-check kernels")
+    ap.add_argument("--regions", type=int, default=0,
+                    help="number of timed regions of --steps decodes (0 = until about a second has been timed, at least 5; "
+                         "1 keeps a profiler capture short)")
     ap.add_argument("--per-step", default=None, help="write a per-step table (name, ms, TFLOP/s, GB/s) to this file")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "vd" else args.warmup
@@ -288,7 +291,7 @@ def main():
         """Regions of `steps` calls back to back until about a second of load has been timed (at least
         five), so that the clock record holds enough samples; the median region is the reported one."""
         first = timed_region(fn, steps)
-        n = max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1))
+        n = args.regions if args.regions > 0 else max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1))
         return [first] + [timed_region(fn, steps) for _ in range(n - 1)]
 
     t_begin = time.time()
@@ -324,7 +327,8 @@ def main():
         sampler2.wait_for_samples(1)
     t2_begin = time.time()
     first = e2e_region()
-    e2e_regions = [first] + [e2e_region() for _ in range(max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1)) - 1)]
+    n_e2e = args.regions if args.regions > 0 else max(5, min(40, int(1000.0 / max(first, 1e-3)) + 1))
+    e2e_regions = [first] + [e2e_region() for _ in range(n_e2e - 1)]
     t2_end = time.time()
     e2e_clocks = sampler2.stop(t2_begin, t2_end) if sampler2 else None
     e2e_ms = sorted(e2e_regions)[len(e2e_regions) // 2] / args.steps
