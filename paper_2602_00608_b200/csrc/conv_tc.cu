@@ -246,7 +246,7 @@ __device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
 template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
-               const __grid_constant__ CUtensorMap tmap_y, unsigned int* status) {
+               const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
     using Cfg = TileCfg<BN, CG, PH>;
     constexpr int NBUF = Cfg::NBUF, PAIR = Cfg::PAIR, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
@@ -264,7 +264,13 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int taps = a.ksize * a.ksize;
     const int kchunks = a.Cin >> 6;
-    const int kchunks2 = a.x2 ? (a.Cin2 >> 6) : 0;          // extra K: 1x1 shortcut on a second input
+    // Extra K: the 1x1 shortcut on a second input (fp32, at the output resolution), in sub-chunks of 32 channels.
+    // It needs no halo and no transform, so it does not go through the producers: a bulk tensor load puts the
+    // fp32 tile (16 x 8 pixels x 32 channels = 128 rows of 128 bytes) straight into an operand stage, the weights
+    // come as fp32 too, and the products are tcgen05.mma kind::tf32 (K = 8) into the same accumulator.  Operands
+    // keep 10 significant bits instead of bf16's 8; the tensor time of these chunks doubles, the producers' is gone.
+    const int kchunks2 = a.x2 ? (a.Cin2 >> 5) : 0;
+    constexpr uint32_t SC_TILE_BYTES = TILE_H * TILE_W * 128;
     const int ktotal = kchunks + kchunks2;
     const int cout_pad = (a.Cout % 128 == 0) ? a.Cout : 16; // rows per tap in the packed weights
     Sched sched;
@@ -397,9 +403,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             auto issue = [&](const Pos& p) -> uint32_t {
                 const bool second = p.kc >= kchunks;
                 const int c0 = (second ? p.kc - kchunks : p.kc) * 64;
-                const bool centre_only = second || a.ksize == 1;
+                const bool centre_only = a.ksize == 1;
                 const Tile& tile = p.tile;
-                if (p.cnt == 0) { cp_async_commit(); return 0u; }  // no tile of this CTA in the item: nothing to copy
+                if (p.cnt == 0 || second) { cp_async_commit(); return 0u; }  // no tile of this CTA in the item, or a shortcut chunk (loaded by TMA): nothing to copy
                 uint32_t vm = 7u;
                 const bool interior = tile.ty0 > 0 && tile.tx0 > 0 && tile.ty0 + TILE_H < a.H && tile.tx0 + TILE_W < a.W;
                 if (interior && !centre_only) {
@@ -428,7 +434,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         vm |= (v ? 1u : 0u) << u;
                     }
                 }
-                if (!second) {
+                {
                     const char* xb = (const char*)a.x
                         + ((((size_t)tile.b * a.Hs + (tile.ty0 >> up)) * a.Ws + (tile.tx0 >> up)) * a.Cin + c0 + (IN_BF16 ? j * 8 : j * 4)) * ESZ;
 #pragma unroll
@@ -437,15 +443,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const char* src = v ? xb + goff[u] : (const char*)a.x;
                         cp_async16(st_lo + (uint32_t)(u * NUM_PRODUCERS * 16), src, v ? 16u : 0u);
                         if (!IN_BF16) cp_async16(st_hi + (uint32_t)(u * NUM_PRODUCERS * 16), src + (v ? 128 : 0), v ? 16u : 0u);
-                    }
-                } else {             // fused shortcut: fp32 input at the output resolution, centre pixels only
-                    const char* xb = (const char*)a.x2 + ((((size_t)tile.b * a.H + tile.ty0) * a.W + tile.tx0) * a.Cin2 + c0 + j * 4) * 4;
-#pragma unroll
-                    for (int u = 0; u < BATCH; ++u) {
-                        const bool v = (vm >> u) & 1u;
-                        const char* src = v ? xb + (((int)(pyx[u] & 0xffu) - 1) * a.W + ((int)((pyx[u] >> 8) & 0xffu) - 1)) * a.Cin2 * 4 : (const char*)a.x2;
-                        cp_async16(st_lo + (uint32_t)(u * NUM_PRODUCERS * 16), src, v ? 16u : 0u);
-                        cp_async16(st_hi + (uint32_t)(u * NUM_PRODUCERS * 16), src + (v ? 128 : 0), v ? 16u : 0u);
                     }
                 }
                 cp_async_commit();
@@ -481,8 +478,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const bool cur_have = cur_cnt > 0;               // without a tile the CTA still follows the barriers
                 const uint32_t cur_vm = vm_next;
                 const bool second = cur_kc >= kchunks;
-                const bool pro = prologue && !second;
-                const bool in_bf16 = IN_BF16 && !second;
+                const bool pro = prologue;
+                constexpr bool in_bf16 = IN_BF16;
                 advance(nx);
                 const bool have_next = nx.t < sched.end;
                 cp_async_wait_all();                             // this thread's pieces of the current unit have landed
@@ -496,11 +493,17 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 if (cur_slot == 0) {
                     ok = mbar_wait(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                     if (!ok) break;
+                    // a shortcut chunk: the stage will be filled by bulk tensor loads (one per tile of this CTA)
+                    if (second && ptid == 0 && cur_have) mbar_expect_tx(smem_u32(&bars->a_full[stage]), (uint32_t)cur_cnt * SC_TILE_BYTES);
                 }
                 uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + cur_slot * A_TILE_BYTES;
+                if (second && ptid == 0 && cur_have) {
+                    const Tile ct = sched.get(sched.index(cur_t, cur_slot), BN);
+                    tma_load_4d(smem_u32(dst_tile), &tmap_x2, (cur_kc - kchunks) * 32, ct.tx0, ct.ty0, ct.b, smem_u32(&bars->a_full[stage]));
+                }
 #pragma unroll
                 for (int u = 0; u < BATCH; ++u) {
-                    if (!cur_have) break;
+                    if (!cur_have || second) break;
                     uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
                     if (cur_vm & (1u << u)) {
                         float v[8];
@@ -518,11 +521,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     if (in_bf16) {
                         *(uint4*)(dst_tile + soff[u]) = make_uint4(o0, o1, o2, o3);
                     } else {
-                        uint32_t so = soff[u];
-                        if (IN_BF16) {                           // fp32 second input of a kernel whose first input is bf16
-                            const uint32_t pix = so >> 7;
-                            so = pix * 128 + (((j >> 1) ^ (pix & 7)) << 4) + (j & 1) * 8;
-                        }
+                        const uint32_t so = soff[u];
                         *(uint2*)(dst_tile + so) = make_uint2(o0, o1);
                         *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
                     }
@@ -543,9 +542,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const int cnt = sched.mine(n);                   // 0: the peer of a two-CTA pair in an odd tail item
             const Tile tile0 = sched.get(cnt > 0 ? sched.index(t, 0) : t, BN);
             for (int kc = 0; kc < ktotal && ok; ++kc) {
-                const bool second = kc >= kchunks;
-                const int c0 = (second ? kc - kchunks : kc) * 64;
-                const bool centre_only = second || a.ksize == 1;
+                const bool second = kc >= kchunks;             // a shortcut chunk: loaded by TMA, nothing to transform
+                const int c0 = kc * 64;
+                const bool centre_only = a.ksize == 1;
                 const bool pro = prologue && !second;
                 float sc[8], sh[8];
                 if (pro) {
@@ -584,30 +583,27 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 vm |= (v ? 1u : 0u) << u;
                             }
                         }
-                        if (!have) vm = 0u;
+                        if (!have || second) vm = 0u;
                         Raw8 raw[BATCH];
-                        if (!second) {
+                        {
                             const char* xb = (const char*)a.x
                                 + ((((size_t)tile.b * a.Hs + (tile.ty0 >> up)) * a.Ws + (tile.tx0 >> up)) * a.Cin + c0 + (IN_BF16 ? j * 8 : j * 4)) * ESZ;
 #pragma unroll
                             for (int u = 0; u < BATCH; ++u)
                                 if (vm & (1u << u)) load_raw_at(IN_BF16, xb + goff[u], raw[u]);
-                        } else {             // fused shortcut: fp32 input at the output resolution, centre pixels only
-                            const char* xb = (const char*)a.x2 + ((((size_t)tile.b * a.H + tile.ty0) * a.W + tile.tx0) * a.Cin2 + c0 + j * 4) * 4;
-#pragma unroll
-                            for (int u = 0; u < BATCH; ++u)
-                                if (vm & (1u << u))
-                                    load_raw_at(false, xb + (((int)(pyx[u] & 0xffu) - 1) * a.W + ((int)((pyx[u] >> 8) & 0xffu) - 1)) * a.Cin2 * 4, raw[u]);
                         }
                         if (slot == 0) {
                             ok = mbar_wait<PH ? 256 : 0>(smem_u32(&bars->a_empty[stage]), phase ^ 1, abort_flag);
                             if (!ok) break;
+                            if (second && ptid == 0 && cnt > 0) mbar_expect_tx(smem_u32(&bars->a_full[stage]), (uint32_t)cnt * SC_TILE_BYTES);
                         }
                         uint8_t* dst_tile = smem_a + stage * A_STAGE_BYTES + slot * A_TILE_BYTES;
-                        const bool in_bf16 = IN_BF16 && !second;
+                        if (second && ptid == 0 && have)
+                            tma_load_4d(smem_u32(dst_tile), &tmap_x2, (kc - kchunks) * 32, tile.tx0, tile.ty0, tile.b, smem_u32(&bars->a_full[stage]));
+                        constexpr bool in_bf16 = IN_BF16;
 #pragma unroll
                         for (int u = 0; u < BATCH; ++u) {
-                            if (!have) break;
+                            if (!have || second) break;
                             uint32_t o0 = 0u, o1 = 0u, o2 = 0u, o3 = 0u;
                             if (vm & (1u << u)) {
                                 float v[8];
@@ -627,11 +623,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             if (in_bf16) {
                                 *(uint4*)(dst_tile + soff[u]) = make_uint4(o0, o1, o2, o3);
                             } else {
-                                uint32_t so = soff[u];
-                                if (IN_BF16) {               // fp32 second input of a kernel whose first input is bf16
-                                    const uint32_t pix = so >> 7;
-                                    so = pix * 128 + (((j >> 1) ^ (pix & 7)) << 4) + (j & 1) * 8;
-                                }
+                                const uint32_t so = soff[u];
                                 *(uint2*)(dst_tile + so) = make_uint2(o0, o1);
                                 *(uint2*)(dst_tile + (so ^ 64u)) = make_uint2(o2, o3);
                             }
@@ -886,10 +878,10 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         }
                     } else {
                         const int rw = min(tl[sl].tx0 + TILE_W, a.W) - tl[sl].tx0, n = rw * (min(tl[sl].ty0 + TILE_H, a.H) - tl[sl].ty0);
-                        const char* base = (const char*)a.x2 + (((size_t)tl[sl].b * a.H * a.W) * a.Cin2 + (kc - kchunks) * 64) * 4;
-                        for (int i = lane; i < n * 2; i += 32) {
-                            const int px = i >> 1, ry = px / rw, rx = px - ry * rw;
-                            prefetch_l2(base + ((size_t)(tl[sl].ty0 + ry) * a.W + (tl[sl].tx0 + rx)) * a.Cin2 * 4 + (i & 1) * 128);
+                        const char* base = (const char*)a.x2 + (((size_t)tl[sl].b * a.H * a.W) * a.Cin2 + (kc - kchunks) * 32) * 4;
+                        for (int i = lane; i < n; i += 32) {
+                            const int ry = i / rw, rx = i - ry * rw;
+                            prefetch_l2(base + ((size_t)(tl[sl].ty0 + ry) * a.W + (tl[sl].tx0 + rx)) * a.Cin2 * 4);
                         }
                     }
                 }
@@ -918,12 +910,12 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                             const uint32_t full = leader_bar(&bars->b_full[stage]);
                             const int row0 = tl.n0 + (int)rank * (BN / 2);
                             mbar_arrive_expect_tx_cluster(full, Cfg::B_STAGE_BYTES);
-                            if (second) tma_load_2d_pair(dst, &tmap2, (kc - kchunks) * 64, row0, full);
+                            if (second) tma_load_2d_pair(dst, &tmap2, (kc - kchunks) * 32, row0, full);
                             else tma_load_2d_pair(dst, &tmap, kc * 64, tap * cout_pad + row0, full);
                         } else {
                             const uint32_t full = smem_u32(&bars->b_full[stage]);
                             mbar_arrive_expect_tx(full, Cfg::B_STAGE_BYTES);
-                            if (second) tma_load_2d(dst, &tmap2, (kc - kchunks) * 64, tl.n0, full);
+                            if (second) tma_load_2d(dst, &tmap2, (kc - kchunks) * 32, tl.n0, full);
                             else tma_load_2d(dst, &tmap, kc * 64, tap * cout_pad + tl.n0, full);
                         }
                         ++issued;
@@ -1041,14 +1033,35 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     __syncwarp();
                     if (++bs == (uint32_t)Cfg::B_STAGES) { bs = 0; bph ^= 1; }
                 };
+                // a shortcut sub-chunk: fp32 operands (dense 128-row tile, eight-row groups 1024 bytes apart; fp32 weight
+                // stage), four kind::tf32 MMAs of K = 8 per tile
+                auto shortcut_step = [&](auto two_c, uint32_t td, uint32_t a_lo) {
+                    constexpr bool TWO = decltype(two_c)::value;
+                    constexpr uint32_t idesc_tf32 = make_idesc_tf32(128, BN);
+                    const uint32_t a_hi_dense = desc_hi(1024, 2);
+                    wait_on(b_full0 + bs * 8u, bph);
+                    const uint32_t b_lo = b_lo0 + bs * (uint32_t)(Cfg::B_STAGE_BYTES >> 4);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_tf32_split_on(td, a_lo + 2 * k, a_hi_dense, b_lo + 2 * k, b_hi, idesc_tf32, 1u, lead);
+                    if (TWO) {
+                        const uint32_t td2 = td + Cfg::ACC_COLS, a2 = a_lo + (A_TILE_BYTES >> 4);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) umma_tf32_split_on(td2, a2 + 2 * k, a_hi_dense, b_lo + 2 * k, b_hi, idesc_tf32, 1u, lead);
+                    }
+                    commit_on(b_empty0 + bs * 8u);
+                    __syncwarp();
+                    if (++bs == (uint32_t)Cfg::B_STAGES) { bs = 0; bph ^= 1; }
+                };
                 auto item = [&](auto two_c, uint32_t td, int buf) {
                     uint32_t acc = 0;                         // the first MMA of an item overwrites the accumulator
 #pragma unroll 1
                     for (int kc = 0; kc < ktotal; ++kc) {
-                        const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
+                        const bool centre = a.ksize == 1;                        // single centre tap
                         wait_on(smem_u32(&bars->a_full[as]), aph);
                         uint32_t a_row = a_lo0 + as * (A_STAGE_BYTES >> 4);
-                        if (!centre) {
+                        if (kc >= kchunks) {
+                            if constexpr (CG == 1) shortcut_step(two_c, td, a_row);       // (always after the main chunks: accumulates)
+                        } else if (!centre) {
 #pragma unroll 1
                             for (int ky = 0; ky < 3; ++ky) {
                                 tap_step(two_c, td, a_row, acc);
@@ -1386,7 +1399,7 @@ cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* 
     cfg.attrs = attr;
     cfg.numAttrs = na;
     return cudaLaunchKernelEx(&cfg, kern, ka, *(const CUtensorMap*)plan.tmap, *(const CUtensorMap*)plan.tmap2,
-                              *(const CUtensorMap*)plan.tmap_y, status);
+                              *(const CUtensorMap*)plan.tmap_y, *(const CUtensorMap*)plan.tmap_x2, status);
 }
 
 // can this device co-schedule the CTA pairs of the two-CTA kernels?  (looked up once per device)
@@ -1404,7 +1417,7 @@ bool conv_tc_supported(const ConvArgs& a) {
     if (a.Cin % 64 != 0 || a.Cin < 64) return false;
     if (!a.bf16_operands) return false;
     if (a.ksize != 1 && a.ksize != 3) return false;
-    if (a.x2 && (a.Cin2 % 64 != 0 || a.Cin2 < 64)) return false;
+    if (a.x2 && (a.Cin2 % 32 != 0 || a.Cin2 < 32 || a.upsample)) return false;
     if (a.upsample == 2)     // phase-collapsed form: 3x3, 128-channel blocks, plain NHWC store
         return a.ksize == 3 && a.Cout % 128 == 0 && !a.out_nchw && !a.residual && !a.x2;
     if (a.Cout % 128 == 0) return !a.out_nchw && !a.out_u8;
@@ -1477,6 +1490,7 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
                     CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
                 return cudaErrorInvalidValue;
         }
+        memcpy(plan->tmap_x2, plan->tmap, sizeof(plan->tmap));
         plan->bn = bn;
         plan->batch = a.B;
         plan->y = a.y;
@@ -1484,10 +1498,29 @@ cudaError_t conv_tc_prepare(const ConvArgs& a, ConvTcPlan* plan) {
         return cudaSuccess;
     }
     if (!encode_weights((CUtensorMap*)plan->tmap, a.w, a.Cin, taps * padded_cout(a.Cout), bn / cg)) return cudaErrorInvalidValue;
+    memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
+    memcpy(plan->tmap_x2, plan->tmap, sizeof(plan->tmap));
     if (a.x2) {
-        if (!encode_weights((CUtensorMap*)plan->tmap2, a.w2, a.Cin2, a.Cout, bn / cg)) return cudaErrorInvalidValue;
-    } else {
-        memcpy(plan->tmap2, plan->tmap, sizeof(plan->tmap));
+        if (cg != 1) return cudaErrorInvalidValue;           // the fused shortcut exists in the one-CTA forms
+        // shortcut weights fp32 [Cout][Cin2] (one box = a weight stage: BN rows of 32 channels = 128 bytes)
+        const cuuint64_t wd[2] = {(cuuint64_t)a.Cin2, (cuuint64_t)a.Cout};
+        const cuuint64_t ws[1] = {(cuuint64_t)a.Cin2 * 4};
+        const cuuint32_t wb[2] = {32, (cuuint32_t)bn};
+        const cuuint32_t one2[2] = {1, 1};
+        if (enc((CUtensorMap*)plan->tmap2, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(a.w2), wd, ws, wb, one2,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+        // shortcut input fp32 NHWC [B][H][W][Cin2]; one box = a tile of 16 x 8 pixels x 32 channels, zero beyond the image
+        const cuuint64_t xd[4] = {(cuuint64_t)a.Cin2, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)std::max(a.B, 1)};
+        const cuuint64_t xs[3] = {(cuuint64_t)a.Cin2 * 4, (cuuint64_t)a.W * a.Cin2 * 4, (cuuint64_t)a.H * a.W * a.Cin2 * 4};
+        const cuuint32_t xb[4] = {32, (cuuint32_t)TILE_W, (cuuint32_t)TILE_H, 1};
+        const cuuint32_t one4[4] = {1, 1, 1, 1};
+        if (enc((CUtensorMap*)plan->tmap_x2, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(a.x2), xd, xs, xb, one4,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+        plan->x2 = a.x2;
     }
     if (!a.out_nchw && !a.out_u8) {
         // output [B][H][W][Cout] as a 4-D tensor (channels innermost); a box is one epilogue warp's quarter (4 rows) of a 128-byte-wide slice of a tile
@@ -1514,6 +1547,7 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
     if (!a.out_nchw && !a.out_u8 && (a.y != plan.y || a.B > plan.batch)) return cudaErrorInvalidValue;   // the output map is bound at prepare time
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
     if ((a.upsample == 2) != (plan.phase != 0)) return cudaErrorInvalidValue;
+    if (a.x2 && a.x2 != plan.x2) return cudaErrorInvalidValue;                               // so is the shortcut's input map
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.phase) {
         if (ib && ob) return launch_one<128, true, 1, 2, true>(a, plan, status, s);

@@ -30,7 +30,7 @@ struct Step {
 
 struct WeightJob {           // repack work done once in vd_create
     std::string name;        // source tensor
-    int kind;                // 0 conv weight (packed), 1 vector -> fp32
+    int kind;                // 0 conv weight (packed), 1 vector -> fp32, 2 matrix [Cout][Cin] -> fp32 (same layout)
     bool tc;
     bool phase;              // tensor-core weights of the phase-collapsed upsampling form
     int Cout, Cin, taps;
@@ -183,9 +183,12 @@ class Planner {
         a.w = ptr<void>(cw.w_off);
         a.bias = ptr<float>(cw.b_off);
         if (!shortcut_name.empty()) {          // only requested when the tensor-core kernel takes this layer
-            ConvW sw = conv_weight({shortcut_name}, Cout, Cin2, 1, true);
-            a.w2 = ptr<void>(sw.w_off);
-            a.bias2 = ptr<float>(sw.b_off);
+            // the fused shortcut multiplies in tf32: its weight stays an fp32 [Cout][Cin2] matrix
+            const size_t w2_off = alloc((size_t)Cout * Cin2 * 4), b2_off = alloc((size_t)Cout * 4);
+            h_->jobs.push_back({shortcut_name + ".weight", 2, false, false, Cout, Cin2, 1, 0, 0, w2_off});
+            h_->jobs.push_back({shortcut_name + ".bias", 1, false, false, Cout, 0, 0, 0, 0, b2_off});
+            a.w2 = ptr<void>(w2_off);
+            a.bias2 = ptr<float>(b2_off);
         }
         s.conv = a;
         s.use_tc = tc;
@@ -231,7 +234,7 @@ class Planner {
                      VD_F32, false, false);
             return;
         }
-        const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 64 == 0;
+        const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 32 == 0;
         if (fuse) {      // the 1x1 shortcut rides along as extra K of conv2: no tensor of its own
             add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, -1, y,
                      VD_F32, false, false, p + ".shortcut", x, Cin);
@@ -569,15 +572,15 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
         if (!t) { std::string m = "missing weight tensor: " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
         if (!t->dptr) { std::string m = "NULL pointer for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
         if (t->dtype != cfg->dtype) { std::string m = "dtype of " + j.name + " differs from config.dtype"; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
-        int64_t want = j.kind == 0 ? (int64_t)j.Cout * j.Cin * j.taps : j.Cout;
+        int64_t want = j.kind == 1 ? j.Cout : (int64_t)j.Cout * j.Cin * j.taps;
         int64_t have = 1;
         if (t->ndim < 1 || t->ndim > 4) { std::string m = "bad ndim for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
         for (int d = 0; d < t->ndim; ++d) have *= t->shape[d];
         bool ok = have == want && t->shape[0] == j.Cout;
-        if (ok && j.kind == 0) ok = t->ndim >= 2 && t->shape[1] == j.Cin;
+        if (ok && j.kind != 1) ok = t->ndim >= 2 && t->shape[1] == j.Cin;
         if (!ok) { std::string m = "shape mismatch for " + j.name; delete h; return fail(nullptr, VD_ERR_INVALID_ARG, m); }
-        if (j.kind == 1) {
-            e = launch_to_f32(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, s);
+        if (j.kind == 1 || j.kind == 2) {
+            e = launch_to_f32(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.kind == 1 ? j.Cout : (int64_t)j.Cout * j.Cin, s);
         } else if (j.tc) {
             e = launch_pack_weight_tc(t->dptr, t->dtype, h->ws + j.dst_off, j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, j.phase, s);
         } else {

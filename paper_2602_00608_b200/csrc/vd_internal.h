@@ -29,7 +29,7 @@ struct ConvArgs {
     int out_u8;             // 1: y is the display-packed frame, NHWC uint8 [B,H,W,Cout] (out_dtype and out_nchw are ignored)
     // optional fused 1x1 shortcut (tensor-core kernel only): y += W2 * x2 + bias2
     const void* x2;         // fp32 NHWC [B,H,W,Cin2] at the output resolution, or null
-    const void* w2;         // packed bf16 [Cout][Cin2]
+    const void* w2;         // fp32 [Cout][Cin2] (tensor-core kernel: the shortcut's products are tf32)
     const float* bias2;     // [Cout] or null
     int Cin2;
     // tensor-core kernel: ceil(2^32 / d) for the divisors of its tile numbering (tiles per image, channel
@@ -105,6 +105,8 @@ struct alignas(64) ConvTcPlan {
     unsigned char tmap[128];
     unsigned char tmap2[128];   // weights of the fused shortcut (copy of tmap when unused)
     unsigned char tmap_y[128];  // output tensor (NHWC outputs leave through bulk tensor stores)
+    unsigned char tmap_x2[128]; // input of the fused shortcut (fp32 NHWC, loaded by TMA)
+    const void* x2;             // the address tmap_x2 was built for
     void* y;                    // the output address tmap_y was built for
     int batch;                  // frames covered by tmap_y
     int bn;
