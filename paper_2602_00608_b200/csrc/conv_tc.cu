@@ -1,8 +1,9 @@
 // Implicit-GEMM 3x3 / 1x1 convolution on the 5th-generation tensor cores (tcgen05 + TMEM), with
 // the paper's fusion folded around it (Section IV-B.1, Eq. 9): the GroupNorm-apply + SiLU of the
-// chain runs in the operand prologue, nearest-2x upsampling is an address computation, and bias,
-// residual add, the 1x1 shortcut and the output cast run in / next to the same accumulation, so
-// each activation crosses HBM once.
+// chain runs in the operand prologue, nearest-2x upsampling is collapsed into four 2x2 convolutions
+// of the source (or, in the 9-tap form, an address computation), and bias, residual add, the 1x1
+// shortcut and the output cast run in / next to the same accumulation, so each activation crosses
+// HBM once.
 //
 // Persistent kernel, one CTA per SM, roles decoupled through mbarrier rings:
 //   * tile = 16x8 output pixels x BN output channels:  D[128 x BN] = sum over taps and 64-channel
@@ -16,8 +17,9 @@
 //     Out-of-image halo pixels are exact zeros (padding applies to the transformed tensor).
 //     For two-tile items and two-CTA pairs the raw input of the next unit is staged in shared
 //     memory by cp.async while the current unit is transformed.
-//     An optional second input (the block's raw input for a width-changing ResNet block) is
-//     appended as extra K with a single centre tap: the 1x1 shortcut without its own round trip.
+//     An optional second input (the block's raw fp32 input for a width-changing ResNet block) is
+//     appended as extra K: the 1x1 shortcut without its own round trip.  It needs no transform, so
+//     bulk tensor loads put it into the operand stages as it is and it is multiplied in tf32.
 //   * 1 warp streams the weights (bf16 [tap][Cout][Cin]) by TMA into 128B-swizzled stages.
 //   * 1 warp issues tcgen05.mma (M=128, N=BN, K=16) into TMEM accumulators, double-buffered so an
 //     item's epilogue overlaps the next item.  The whole warp runs the loop and the tensor
@@ -30,8 +32,9 @@
 //     is done once, by the memory system), so the residual never passes through the SM.
 //     The 3-channel frame head writes its NCHW planes directly.
 //   * 1 warp asks L2 ahead of time for the input lines of coming chunks.
-//   * Upsampling layers with 256-channel blocks run as pairs of CTAs (tcgen05.mma.cta_group::2,
-//     see TileCfg).
+//   * Upsampling layers run as pairs of CTAs (tcgen05.mma.cta_group::2) in the phase-collapsed
+//     form: one halo tile of 16x8 SOURCE pixels, four parity accumulators, 16 instead of 36 tap
+//     products (see TileCfg and PhaseSched).
 // Every wait is bounded: on expiry the CTA records a code in the status word and unwinds.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -93,7 +96,8 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
     static constexpr int PAIR = PH ? 1 : (BN == 256 ? 1 : 2);        // tiles per work item (and CTA)
     static constexpr int B_STAGE_BYTES = (PH ? 2 : 1) * (BN / CG) * 128;   // this CTA's rows x 64 bf16 (phase: two taps)
-    static constexpr int OUT_BUFS = (PH || BN == 128) ? 2 : 1;   // 128-channel blocks: a second slice buffer pays more than a fourth weight stage                      // output slices per epilogue warp
+    // output slices per epilogue warp (128-channel blocks: a second slice buffer pays more than a fourth weight stage)
+    static constexpr int OUT_BUFS = (PH || BN == 128) ? 2 : 1;
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
     static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? 3 : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
