@@ -149,6 +149,26 @@ def test_full_size_configs_whole_frame_against_the_oracle(env, idx):
     assert r2 <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
 
 
+@pytest.mark.parametrize("h,w,b", [(1, 1, 1), (2, 3, 2), (5, 4, 3), (33, 47, 2)])
+def test_sdvae_bf16_degenerate_and_odd_sizes(env, h, w, b):
+    """Latents smaller than one tile (every tile of every level ragged, most of each halo outside the image), and a
+    larger odd size: the tensor-core path against the FFMA path on every pixel, and against the oracle where
+    the oracle finishes in seconds."""
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[2]
+    z = synth.workload_latents(wl, batch=b, h=h, w=w)
+    dec, got, wts = _decode(env, wl, z)
+    dec2, got2, _ = _decode(env, wl, z, flags=vd.VD_FLAG_FORCE_SIMT)
+    assert got.shape == (b, 3, 8 * h, 8 * w)
+    d = got.float() - got2.float()
+    assert float(d.norm() / got2.float().norm()) <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
+    if h * w <= 20:
+        want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
+        g = got.float().cpu().numpy()
+        assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+    dec.check_status()
+
+
 def test_platformer_shape_256x256_stream_against_the_oracle(env):
     """The paper's second workload shape (256x256 frames, latent 32x32), four AR(1) frames in one batch:
     every pixel of the first and last frame against the oracle run in the test."""
