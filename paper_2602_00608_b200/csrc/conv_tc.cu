@@ -699,6 +699,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             uint8_t* wout = smem_out + ew * (Cfg::OUT_BUFS * WARP_SLICE_BYTES);
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
             int bias_n0 = -1;
+            const uint64_t pol_out = l2_policy_evict_last();
             constexpr int TAIL_BUFS = Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) >= 2 ? Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) : 2;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int n = sched.count(t);
@@ -813,9 +814,9 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                 constexpr int CS = 32 * PPS;
                                 // phase form: the tile is one parity of a 32x16 output block: rows 2i + a through the map of
                                 // row parity a (tmap_y, tmap2), columns 2j + b through the map's parity coordinate
-                                if (PH) tma_store_5d((slot >> 1) ? &tmap2 : &tmap_y, smem_u32(obuf), tl.n0 + sl * CS, slot & 1, tl.tx0, tl.ty0 + 4 * ew, tl.b);
-                                else if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
-                                else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b);
+                                if (PH) tma_store_5d((slot >> 1) ? &tmap2 : &tmap_y, smem_u32(obuf), tl.n0 + sl * CS, slot & 1, tl.tx0, tl.ty0 + 4 * ew, tl.b, pol_out);
+                                else if (reduce_add) tma_reduce_add_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b, pol_out);
+                                else tma_store_4d(&tmap_y, smem_u32(obuf), tl.n0 + sl * CS, tl.tx0, tl.ty0 + 4 * ew, tl.b, pol_out);
                                 bulk_commit_group();
                             }
                         }

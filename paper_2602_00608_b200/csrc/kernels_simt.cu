@@ -75,6 +75,25 @@ template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bflo
     v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
 }
 
+// Streaming loads of the statistics pass: a line it brings in is the first to leave L2 again, so the lines the
+// producing kernel has just written stay resident until the pass reaches them.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+template <typename T> __device__ __forceinline__ void load4_stream(const T* p, float v[4], uint64_t pol);
+template <> __device__ __forceinline__ void load4_stream<float>(const float* p, float v[4], uint64_t pol) {
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]) : "l"(p), "l"(pol));
+}
+template <> __device__ __forceinline__ void load4_stream<__nv_bfloat16>(const __nv_bfloat16* p, float v[4], uint64_t pol) {
+    uint2 t;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.u32 {%0, %1}, [%2], %3;" : "=r"(t.x), "=r"(t.y) : "l"(p), "l"(pol));
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xffff0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
 constexpr int kGnThreads = 512;
 constexpr int kGnFinalLoads = (kGnMaxChunks + 15) / 16;   // records a thread of the last block reads in one round (32 groups: 16 slices)
 
@@ -101,10 +120,11 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
         load4<T>(x + (size_t)(a.P / 2) * a.C + (slot * 4 / cpg) * cpg, kv);
         const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
         int p = p0 + row;
+        const uint64_t pol = policy_evict_first();
         for (; p + (U - 1) * rows < p1; p += U * rows) {        // U independent loads in flight
             float u[U][4];
 #pragma unroll
-            for (int j = 0; j < U; ++j) load4<T>(x + (size_t)(p + j * rows) * a.C + slot * 4, u[j]);
+            for (int j = 0; j < U; ++j) load4_stream<T>(x + (size_t)(p + j * rows) * a.C + slot * 4, u[j], pol);
 #pragma unroll
             for (int j = 0; j < U; ++j)
 #pragma unroll
