@@ -30,8 +30,8 @@
 //     traffic and clip the ragged image edge.  Where the layer has a residual, the output buffer
 //     IS the residual stream and the store is a bulk tensor reduce-add (the fp32 add x + conv(h)
 //     is done once, by the memory system), so the residual never passes through the SM.
-//     The 3-channel frame head writes its NCHW planes directly.
-//   * 1 warp asks L2 ahead of time for the input lines of coming chunks.
+//     The 3-channel frame head writes its NCHW planes directly.  Outputs are stored with the
+//     evict-last L2 policy: the statistics pass and the layer that follow read them from L2.
 //   * Upsampling layers run as pairs of CTAs (tcgen05.mma.cta_group::2) in the phase-collapsed
 //     form: one halo tile of 16x8 SOURCE pixels, four parity accumulators, 16 instead of 36 tap
 //     products (see TileCfg and PhaseSched).
@@ -826,72 +826,6 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 t += n;
             }
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
-        }
-    } else if (warp == PREFETCH_WARP) {
-        // ------------------------------------------------ input prefetch into L2
-        // The activations of the large layers do not fit the L2 cache, and a producer thread can
-        // keep only one unit of loads in flight in its registers, which does not cover the latency
-        // of device memory.  This warp follows the producers' progress on the operand barriers and
-        // asks L2, PF_AHEAD chunks ahead of them, for the 64-channel pixel records the chunk's
-        // tiles will read (one prefetch per 128-byte line; bulk prefetches of such small ranges
-        // would crowd the copy engine that also brings the weights).  It is best effort: a wait that
-        // runs out ends the role quietly.
-        griddep_wait();
-        constexpr int PF_AHEAD = 2;
-        const int esz = IN_BF16 ? 2 : 4;
-        const int h = a.ksize == 3 ? 1 : 0;
-        const int up = a.upsample ? 1 : 0;
-        int waited = 0;                                      // chunks of the CTA whose completion has been observed
-        int q = 0;                                           // chunk being prefetched (counted over the CTA's work)
-        bool ok = true;
-        // progress is read from the operand "full" barriers; in the two-CTA form those live in the leader
-        // only, so there it is read from the "empty" barriers (chunks consumed), A_STAGES chunks later
-        constexpr int PF_LEAD = CG == 2 ? PF_AHEAD + Cfg::A_STAGES : PF_AHEAD;
-        for (int t = sched.begin; t < sched.end && ok;) {
-            const int n = sched.count(t);
-            const int cnt = sched.mine(n);
-            Tile tl[PAIR];
-#pragma unroll
-            for (int sl = 0; sl < PAIR; ++sl) tl[sl] = sched.get(sl < cnt ? sched.index(t, sl) : t, BN);
-            for (int kc = 0; kc < ktotal && ok; ++kc, ++q) {
-                while (waited < q - PF_LEAD + 1 && ok) {    // stay at most PF_LEAD chunks ahead
-                    const uint32_t bar = smem_u32(CG == 2 ? &bars->a_empty[waited % Cfg::A_STAGES] : &bars->a_full[waited % Cfg::A_STAGES]);
-                    const uint32_t par = (uint32_t)(waited / Cfg::A_STAGES) & 1u;
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(bar, par)) {
-                        __nanosleep(200);
-                        if (*abort_flag || clock64() - t0 > 400000) { ok = false; break; }
-                    }
-                    ++waited;
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const bool second = kc >= kchunks;
-#pragma unroll
-                for (int sl = 0; sl < PAIR; ++sl) {
-                    if (sl >= cnt) continue;
-                    if (!second) {
-                        const int y0 = max(tl[sl].ty0 - h, 0) >> up, y1 = (min(tl[sl].ty0 + TILE_H + h, a.H) - 1) >> up;
-                        const int x0 = max(tl[sl].tx0 - h, 0) >> up, x1 = (min(tl[sl].tx0 + TILE_W + h, a.W) - 1) >> up;
-                        const int rw = x1 - x0 + 1, n = rw * (y1 - y0 + 1);
-                        const char* base = (const char*)a.x + (((size_t)tl[sl].b * a.Hs * a.Ws) * a.Cin + kc * 64) * esz;
-                        const int lpp = IN_BF16 ? 1 : 2;            // 128-byte lines per pixel record
-                        for (int i = lane; i < n * lpp; i += 32) {
-                            const int px = IN_BF16 ? i : i >> 1, ln = IN_BF16 ? 0 : i & 1;
-                            const int ry = px / rw, rx = px - ry * rw;
-                            prefetch_l2(base + ((size_t)(y0 + ry) * a.Ws + (x0 + rx)) * a.Cin * esz + ln * 128);
-                        }
-                    } else {
-                        const int rw = min(tl[sl].tx0 + TILE_W, a.W) - tl[sl].tx0, n = rw * (min(tl[sl].ty0 + TILE_H, a.H) - tl[sl].ty0);
-                        const char* base = (const char*)a.x2 + (((size_t)tl[sl].b * a.H * a.W) * a.Cin2 + (kc - kchunks) * 32) * 4;
-                        for (int i = lane; i < n; i += 32) {
-                            const int ry = i / rw, rx = i - ry * rw;
-                            prefetch_l2(base + ((size_t)(tl[sl].ty0 + ry) * a.W + (tl[sl].tx0 + rx)) * a.Cin2 * 4);
-                        }
-                    }
-                }
-            }
-            t += n;
         }
     } else if (warp == TMA_WARP) {
         // ------------------------------------------------ weight loads (TMA)

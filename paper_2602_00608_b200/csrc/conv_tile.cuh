@@ -22,10 +22,9 @@ static_assert(BATCH * NUM_PRODUCERS == ITEMS, "producer threads must tile the ha
 // MMA-issuing thread no priority: measured, fifteen warps of dense arithmetic stretch its
 // wait / 4 x MMA / commit sequence from 513 to about 1800 cycles, while the same warps kept off its
 // sub-partition cost nothing.  So sub-partition 0 carries only the MMA warp, the TMA warp and one
-// epilogue warp (warp 12 prefetches inputs into L2; warps 8 and 20 idle until the end), and the fifteen producer warps are the
+// epilogue warp (warps 8, 12 and 20 idle until the end), and the fifteen producer warps are the
 // warps with warp % 4 != 0 outside the epilogue: five per remaining sub-partition.
 constexpr int MMA_WARP = 0;
-constexpr int PREFETCH_WARP = 12;                                   // asks L2 for the next item's input rows
 constexpr int TMA_WARP = 4;
 constexpr int EPI_WARP0 = 16;                                        // warps 16-19 (warp % 4 = TMEM lane quarter)
 constexpr int NUM_THREADS = 24 * 32;
