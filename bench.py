@@ -203,6 +203,8 @@ def main():
     ap.add_argument("--impl", default="vd", choices=["vd", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="force the FFMA cross-check kernels")
+    ap.add_argument("--fused-stats", action="store_true",
+                    help="GroupNorm statistics in the producing convolution's epilogue where it can (VD_FLAG_FUSED_STATS; default: a pass of their own)")
     ap.add_argument("--regions", type=int, default=0,
                     help="number of timed regions of --steps decodes (0 = until about a second has been timed, at least 5; "
                          "1 keeps a profiler capture short)")
@@ -243,7 +245,8 @@ def main():
     peaks = load_peaks()
     wts = synth.workload_weights(wl)
     dec = binding.Decoder(wl.arch, wl.dtype, wl.latent_h, wl.latent_w, wl.batch, wl.groups, wl.eps, wts,
-                          binding.VD_FLAG_FORCE_SIMT if args.simt else 0, device=dev)
+                          (binding.VD_FLAG_FORCE_SIMT if args.simt else 0) |
+                          (binding.VD_FLAG_FUSED_STATS if args.fused_stats else 0), device=dev)
     z_np = synth.workload_latents(wl)
     z = torch.from_numpy(z_np).to(dev, dec.dtype)
     frames = torch.empty((wl.batch,) + dec.out_shape, dtype=dec.dtype, device=dev)

@@ -45,6 +45,9 @@ typedef struct {
     int32_t phase_collapsed;    /* 1: an upsampling conv run as four 2x2 convolutions of the source (flops_per_frame
                                    still counts the layer's own 9 taps; the kernel executes 4/9 of them) */
     int32_t out_u8;             /* 1: the output is the display-packed uint8 NHWC frame (VD_FLAG_OUT_U8) */
+    int32_t stats_fused;        /* 1: a convolution whose epilogue also produces the statistics (scale, shift) of the
+                                   GroupNorm that follows; that GroupNorm has no step of its own then */
+    int32_t reserved;
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);
@@ -112,6 +115,21 @@ VD_API vd_status vd_conv_pack_weight(const vd_conv_desc* d, const void* w_oihw, 
 VD_API vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* w_packed, const float* bias,
                               const float* scale, const float* shift, const float* residual, void* y,
                               void* cuda_stream);
+
+/* vd_op_conv2d and, from the same launch, the statistics of GroupNorm(y) folded with the affine parameters
+ * (Section IV-B.1: the normalisation's reduction is taken while the tile is on chip):
+ *   out_scale[n,c] = gamma[c]*rstd[n,g], out_shift[n,c] = beta[c] - mean[n,g]*out_scale[n,c]   (device fp32 [batch,c_out]),
+ * mean and biased variance of the fp32 values before they are rounded to y's dtype.  Tensor-core kernel only:
+ * c_out % 128 == 0, bf16 NHWC output, no residual, no upsampling of kind 2, groups <= 32 holding 4, 8 or 16 channels
+ * each; anything else returns VD_ERR_UNSUPPORTED.  `scratch`: device memory of vd_conv_stats_scratch_bytes bytes
+ * (the per-group sums, then an arrival counter; the call clears both itself).  Totals of a tile are turned into
+ * 64-bit fixed point (2^-20 for sums, 2^-16 for sums of squares) and all further additions are integer
+ * additions: results are bitwise reproducible and do not depend on the batch. */
+VD_API size_t vd_conv_stats_scratch_bytes(int32_t batch, int32_t groups);
+VD_API vd_status vd_op_conv2d_stats(const vd_conv_desc* d, const void* x, const void* w_packed, const float* bias,
+                                    const float* scale, const float* shift, void* y, int32_t groups, float eps,
+                                    const float* gamma, const float* beta, float* out_scale, float* out_shift,
+                                    void* scratch, void* cuda_stream);
 
 /* GroupNorm statistics of x (device NHWC [batch,h,w,c], dtype `dtype`) folded with the affine
  * parameters: scale[n,c] = gamma[c]*rstd[n,g], shift[n,c] = beta[c] - mean[n,g]*scale[n,c]

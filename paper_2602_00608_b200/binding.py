@@ -18,6 +18,7 @@ VD_FLAG_FORCE_SIMT = 0x1
 VD_FLAG_UPSAMPLE_9TAP = 0x2
 VD_FLAG_OUT_U8 = 0x4
 VD_FLAG_CANARY = 0x8
+VD_FLAG_FUSED_STATS = 0x10
 VD_IMPL_AUTO, VD_IMPL_SIMT, VD_IMPL_TC = 0, 1, 2
 VD_STEP_INGEST, VD_STEP_GN_STATS, VD_STEP_CONV, VD_STEP_ATTENTION = 0, 1, 2, 3
 STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", -3: "VD_ERR_WORKSPACE",
@@ -26,7 +27,7 @@ STATUS_NAMES = {0: "VD_OK", -1: "VD_ERR_INVALID_ARG", -2: "VD_ERR_UNSUPPORTED", 
 EXPORTED = [
     "vd_query_workspace", "vd_create", "vd_decode", "vd_decode_extrapolated", "vd_decode_host", "vd_get_status",
     "vd_last_error", "vd_destroy", "vd_num_steps", "vd_get_step", "vd_profile", "vd_debug_stop_after",
-    "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_gn_scratch_bytes", "vd_op_gn_stats",
+    "vd_conv_packed_weight_bytes", "vd_conv_pack_weight", "vd_op_conv2d", "vd_conv_stats_scratch_bytes", "vd_op_conv2d_stats", "vd_gn_scratch_bytes", "vd_op_gn_stats",
     "vd_op_attention", "vd_attention_scratch_bytes", "vd_op_gn_stats_static", "vd_clear_status", "vd_decode_host_stream", "vd_debug_check_canaries", "vd_debug_status_offset", "vd_debug_wait_probe",
 ]
 
@@ -47,7 +48,8 @@ class VdStepInfo(Structure):
                 ("out_h", c_int32), ("out_w", c_int32), ("out_channels", c_int32), ("out_dtype", c_int32),
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
                 ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
-                ("has_residual", c_int32), ("phase_collapsed", c_int32), ("out_u8", c_int32)]
+                ("has_residual", c_int32), ("phase_collapsed", c_int32), ("out_u8", c_int32),
+                ("stats_fused", c_int32), ("reserved", c_int32)]
 
 
 class VdConvDesc(Structure):
@@ -95,6 +97,9 @@ def lib():
         l.vd_conv_packed_weight_bytes.argtypes = [POINTER(VdConvDesc), POINTER(c_size_t)]
         l.vd_conv_pack_weight.argtypes = [POINTER(VdConvDesc), vp, c_int32, vp, vp]
         l.vd_op_conv2d.argtypes = [POINTER(VdConvDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+        l.vd_conv_stats_scratch_bytes.argtypes = [c_int32, c_int32]
+        l.vd_conv_stats_scratch_bytes.restype = c_size_t
+        l.vd_op_conv2d_stats.argtypes = [POINTER(VdConvDesc), vp, vp, vp, vp, vp, vp, c_int32, c_float, vp, vp, vp, vp, vp, vp]
         l.vd_gn_scratch_bytes.argtypes = [c_int32, c_int32]
         l.vd_gn_scratch_bytes.restype = c_size_t
         l.vd_op_gn_stats.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp, vp]
@@ -323,6 +328,32 @@ def op_conv2d(x_nhwc, w_oihw, bias=None, scale=None, shift=None, residual=None, 
         assert t is None or (t.dtype == torch.float32 and t.is_contiguous())
     _check(lib().vd_op_conv2d(byref(d), p(x_nhwc.contiguous()), p(packed), p(bias), p(scale), p(shift), p(residual), p(y), _stream_ptr()))
     return y
+
+
+def op_conv2d_stats(x_nhwc, w_oihw, gamma, beta, groups: int, eps: float, bias=None, scale=None, shift=None, *,
+                    silu=False, out_dtype=None, impl=VD_IMPL_TC):
+    """op_conv2d (bf16 operands, NHWC output) whose epilogue also takes the statistics of GroupNorm(y):
+    returns (y, out_scale, out_shift)."""
+    import torch
+    b, h, w, cin = x_nhwc.shape
+    cout, _, k, _ = w_oihw.shape
+    od = VD_BF16 if out_dtype is None else out_dtype
+    d = conv_desc(b, h, w, cin, cout, k, False, silu, _dt(x_nhwc), od, False, True, impl)
+    nb = c_size_t(0)
+    _check(lib().vd_conv_packed_weight_bytes(byref(d), byref(nb)))
+    packed = torch.empty(nb.value, dtype=torch.uint8, device=x_nhwc.device)
+    w_oihw = w_oihw.contiguous()
+    _check(lib().vd_conv_pack_weight(byref(d), c_void_p(w_oihw.data_ptr()), _dt(w_oihw), c_void_p(packed.data_ptr()), _stream_ptr()))
+    y = torch.empty((b, h, w, cout), dtype=_torch_dtype(od), device=x_nhwc.device)
+    out_scale = torch.empty((b, cout), dtype=torch.float32, device=x_nhwc.device)
+    out_shift = torch.empty((b, cout), dtype=torch.float32, device=x_nhwc.device)
+    scratch = torch.empty(max(1, lib().vd_conv_stats_scratch_bytes(max(b, 1), groups)), dtype=torch.uint8, device=x_nhwc.device)
+    p = lambda t: None if t is None else c_void_p(t.data_ptr())
+    for t in (bias, scale, shift, gamma, beta):
+        assert t is None or (t.dtype == torch.float32 and t.is_contiguous())
+    _check(lib().vd_op_conv2d_stats(byref(d), p(x_nhwc.contiguous()), p(packed), p(bias), p(scale), p(shift), p(y), groups, eps,
+                                    p(gamma), p(beta), p(out_scale), p(out_shift), p(scratch), _stream_ptr()))
+    return y, out_scale, out_shift
 
 
 def op_gn_stats(x_nhwc, gamma, beta, groups: int, eps: float):

@@ -123,6 +123,7 @@ struct Bars {                    // lives in shared memory
     uint64_t acc_full[4], acc_empty[4];
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t stat_last;          // this CTA is the last to finish (it folds the statistics records)
 };
 
 // Tiles are numbered (frame, channel block, tile row, tile column), column fastest.  Every CTA
@@ -243,6 +244,89 @@ __device__ __forceinline__ void tmem_alloc2(uint32_t smem_dst, uint32_t ncols) {
 }
 __device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// ---- GroupNorm statistics of the output, taken in the epilogue (Section IV-B.1: the normalisation's reduction
+// rides on the tensor that is already on chip instead of reading it back from memory).
+// An epilogue thread holds 32 consecutive channels of one pixel per pass.  It adds the values and their squares in
+// quads of four channels, and a transposing butterfly over the warp's 32 pixels leaves the total of value
+// i = lane >> 1 (i < 8: sum of quad i; i >= 8: sum of squares of quad i - 8) in every lane: 15 exchanges instead of
+// 16 full reductions.  The first exchange pairs a quad's sum with its own sum of squares, so it runs quad by quad
+// while the pass is still being converted and stored.
+// The total of a (tile, pass) depends on the tile's values alone.  It is turned into 64-bit fixed point there and
+// then, and every later addition (over the tiles of a CTA, over the CTAs by atomic adds, in the fold) is an
+// integer addition: the result does not depend on how the tiles are divided among the CTAs, on the batch a frame
+// is decoded in, or on the order the atomic adds arrive in.
+constexpr float kStatSumFix = 1048576.f;      // 2^20: sums        (|total| < 2^43 * 2^20 units ... values to about 1e6 in magnitude)
+constexpr float kStatSqFix = 65536.f;         // 2^16: sums of squares (values to about 1e4 in magnitude over 1.4e6 elements)
+__device__ __forceinline__ float stat_quad_first(float a0, float a1, float a2, float a3, bool valid, bool hi) {
+    float s = (a0 + a1) + (a2 + a3);
+    float q = fmaf(a0, a0, fmaf(a1, a1, fmaf(a2, a2, a3 * a3)));
+    s = valid ? s : 0.f;
+    q = valid ? q : 0.f;
+    const float keep = hi ? q : s, send = hi ? s : q;
+    return keep + __shfl_xor_sync(0xffffffffu, send, 16);
+}
+__device__ __forceinline__ long long stat_reduce(float (&v)[8], int lane) {
+#pragma unroll
+    for (int st = 0; st < 3; ++st) {
+        const int half = 4 >> st, bit = 8 >> st;
+        const bool hi = (lane & bit) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const float keep = hi ? v[i + half] : v[i];
+            const float send = hi ? v[i] : v[i + half];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, bit);
+        }
+    }
+    const float r = v[0] + __shfl_xor_sync(0xffffffffu, v[0], 1);
+    return __float2ll_rn(r * ((lane & 16) ? kStatSqFix : kStatSumFix));
+}
+
+// Adds a warp's accumulated pass totals of channel block [n0, n0 + 32 * NP) of frame b to the layer's sums
+// stat_sum[b][group][2] (sum, sum of squares).
+template <int NP>
+__device__ __forceinline__ void stat_flush(const ConvArgs& a, long long (&acc)[NP], int b, int n0, int lane) {
+    const int cpg = a.Cout / a.stat_G;
+    const int vi = lane >> 1, quad = vi & 7, is_q = vi >> 3;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        if ((lane & 1) == 0) {
+            const int g = (n0 + p * 32 + quad * 4) / cpg;
+            atomicAdd(a.stat_sum + ((size_t)b * a.stat_G + g) * 2 + is_q, (unsigned long long)acc[p]);
+        }
+        acc[p] = 0;
+    }
+}
+
+// The CTA that finishes last turns the sums into the affine map of the normalisation (scale = gamma * rstd,
+// shift = beta - mean * scale) and clears them for the next launch.
+__device__ void stat_finalize(const ConvArgs& a, int tid, void* smem_scratch) {
+    float* s_mean = (float*)smem_scratch;
+    float* s_rstd = s_mean + 32;
+    const int G = a.stat_G, cpg = a.Cout / G;
+    for (int b = 0; b < a.B; ++b) {
+        if (tid < G) {
+            unsigned long long* p = a.stat_sum + ((size_t)b * G + tid) * 2;
+            const double S = (double)(long long)__ldcg(p) * (1.0 / (double)kStatSumFix);
+            const double Q = (double)(long long)__ldcg(p + 1) * (1.0 / (double)kStatSqFix);
+            p[0] = 0ull;
+            p[1] = 0ull;
+            const double inv_n = 1.0 / ((double)a.H * (double)a.W * (double)cpg);
+            const double mean = S * inv_n;
+            const double var = fmax(Q * inv_n - mean * mean, 0.0);
+            s_mean[tid] = (float)mean;
+            s_rstd[tid] = 1.0f / sqrtf((float)(var + (double)a.stat_eps));
+        }
+        __syncthreads();
+        for (int c = tid; c < a.Cout; c += NUM_THREADS) {
+            const int gc = c / cpg;
+            const float sc = __ldg(a.stat_gamma + c) * s_rstd[gc];
+            a.stat_scale[(size_t)b * a.Cout + c] = sc;
+            a.stat_shift[(size_t)b * a.Cout + c] = __ldg(a.stat_beta + c) - s_mean[gc] * sc;
+        }
+        __syncthreads();
+    }
 }
 
 // OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC (both through shared memory and TMA stores),
@@ -700,6 +784,13 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
             int bias_n0 = -1;
             const uint64_t pol_out = l2_policy_evict_last();
+            // statistics for the normalisation that follows: per-pass totals of the current (frame, channel block) run
+            constexpr int NPS = NP > 0 ? NP : 1;
+            const bool stats = OUT_MODE == 1 && !PH && NP > 0 && a.stat_sum != nullptr;
+            long long sacc[NPS];
+#pragma unroll
+            for (int p = 0; p < NPS; ++p) sacc[p] = 0;
+            int stat_b = -1, stat_n0 = 0;
             constexpr int TAIL_BUFS = Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) >= 2 ? Cfg::SMEM_B / (4 * WARP_SLICE_BYTES) : 2;
             for (int t = sched.begin; t < sched.end && ok; ++n_item) {
                 const int n = sched.count(t);
@@ -733,6 +824,15 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         }
                     }
                     const Tile tl = sched.get(sched.index(t, PH ? 0 : slot), BN);
+                    bool stat_valid = true;
+                    if (stats) {
+                        if (tl.b != stat_b || tl.n0 != stat_n0) {
+                            if (stat_b >= 0) stat_flush<NPS>(a, sacc, stat_b, stat_n0, lane);
+                            stat_b = tl.b; stat_n0 = tl.n0;
+                        }
+                        const int m = ew * 32 + lane;
+                        stat_valid = tl.ty0 + (m >> 3) < a.H && tl.tx0 + (m & 7) < a.W;
+                    }
                     if (tl.n0 != bias_n0) {                   // (re)load bias (+ shortcut bias) of this channel block
                         __syncwarp();
                         for (int i = lane; i < BN; i += 32)
@@ -780,15 +880,23 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                                                 __uint_as_float(rc[4 * c + 2]) + tb.z, __uint_as_float(rc[4 * c + 3]) + tb.w);
                             }
                         } else {
+                            float v[8];
+                            const bool stat_hi = (lane & 16) != 0;
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
                                 const float4 t0 = bp[2 * c], t1 = bp[2 * c + 1];
+                                const float f[8] = {__uint_as_float(rc[8 * c]) + t0.x, __uint_as_float(rc[8 * c + 1]) + t0.y,
+                                                    __uint_as_float(rc[8 * c + 2]) + t0.z, __uint_as_float(rc[8 * c + 3]) + t0.w,
+                                                    __uint_as_float(rc[8 * c + 4]) + t1.x, __uint_as_float(rc[8 * c + 5]) + t1.y,
+                                                    __uint_as_float(rc[8 * c + 6]) + t1.z, __uint_as_float(rc[8 * c + 7]) + t1.w};
                                 *(uint4*)(orow + (((h * 4 + c) ^ (lane & 7)) << 4)) =
-                                    make_uint4(pack_bf16(__uint_as_float(rc[8 * c]) + t0.x, __uint_as_float(rc[8 * c + 1]) + t0.y),
-                                               pack_bf16(__uint_as_float(rc[8 * c + 2]) + t0.z, __uint_as_float(rc[8 * c + 3]) + t0.w),
-                                               pack_bf16(__uint_as_float(rc[8 * c + 4]) + t1.x, __uint_as_float(rc[8 * c + 5]) + t1.y),
-                                               pack_bf16(__uint_as_float(rc[8 * c + 6]) + t1.z, __uint_as_float(rc[8 * c + 7]) + t1.w));
+                                    make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                                if (stats) {
+                                    v[2 * c] = stat_quad_first(f[0], f[1], f[2], f[3], stat_valid, stat_hi);
+                                    v[2 * c + 1] = stat_quad_first(f[4], f[5], f[6], f[7], stat_valid, stat_hi);
+                                }
                             }
+                            if (stats) sacc[p] += stat_reduce(v, lane);
                         }
                         if (PAIRED && (p & 1) && p + 1 < NP) {           // both buffers are free again: the next two passes
                             tmem_ld32(tacc + (uint32_t)((p + 1) * 32), ra);
@@ -825,6 +933,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 }
                 t += n;
             }
+            if (stats && stat_b >= 0) stat_flush<NPS>(a, sacc, stat_b, stat_n0, lane);
+            if (stats) __threadfence();
             if (lane == 0) bulk_wait_group<0>();             // all stores have landed before the CTA retires
         }
     } else if (warp == TMA_WARP) {
@@ -1164,6 +1274,21 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         if (CG == 2) tmem_dealloc2(tmem_base, (uint32_t)Cfg::TMEM_COLS);
         else tmem_dealloc(tmem_base, (uint32_t)Cfg::TMEM_COLS);
     }
+    if (OUT_MODE != 2 && a.stat_sum) {
+        // every sum of this CTA has been added (and fenced) before the barrier above
+        if (tid == 0) {
+            __threadfence();
+            bars->stat_last = atomicAdd(a.stat_counter, 1u) == gridDim.x - 1u ? 1u : 0u;
+        }
+        __syncthreads();
+        const bool last = bars->stat_last != 0u;
+        __syncthreads();
+        if (last) {
+            __threadfence();
+            stat_finalize(a, tid, smem);
+            if (tid == 0) *a.stat_counter = 0u;              // ready for the next launch
+        }
+    }
 }
 
 // pack OIHW -> bf16 [tap][cout_pad][Cin]
@@ -1363,6 +1488,16 @@ bool conv_tc_supported(const ConvArgs& a) {
     return a.Cout <= 16 && (a.out_nchw || a.out_u8) && !a.residual && !a.x2;      // the frame head: Cout padded to 16
 }
 
+// Layers whose epilogue can take the statistics of the following GroupNorm: the tile passes through the epilogue's
+// registers as its final value (no residual added by the memory system), 32 groups at most, groups of 4, 8 or 16 channels.
+bool conv_tc_stats_supported(const ConvArgs& a, int groups) {
+    if (!conv_tc_supported(a) || a.Cout % 128 != 0 || a.upsample == 2 || a.residual) return false;
+    if (a.out_dtype != VD_BF16) return false;
+    if (groups < 1 || groups > 32 || a.Cout % groups != 0) return false;
+    const int cpg = a.Cout / groups;
+    return cpg == 4 || cpg == 8 || cpg == 16;
+}
+
 bool conv_tc_pairs_available() { return pairs_available(); }
 
 size_t conv_tc_packed_bytes(int Cout, int Cin, int taps, bool phase) {
@@ -1487,6 +1622,8 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
     if (a.residual && a.residual != a.y) return cudaErrorInvalidValue;                      // residual is accumulated in place
     if ((a.upsample == 2) != (plan.phase != 0)) return cudaErrorInvalidValue;
     if (a.x2 && a.x2 != plan.x2) return cudaErrorInvalidValue;                               // so is the shortcut's input map
+    if (a.stat_sum && (!conv_tc_stats_supported(a, a.stat_G) || !a.stat_counter || !a.stat_scale || !a.stat_shift || !a.stat_gamma || !a.stat_beta))
+        return cudaErrorInvalidValue;
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     if (plan.phase) {
         if (ib && ob) return launch_one<128, true, 1, 2, true>(a, plan, status, s);

@@ -54,7 +54,7 @@ struct vd_handle_s {
     std::vector<size_t> guards;          // offsets of the guard regions (VD_FLAG_CANARY)
     std::string err;
     int stop_after = -1;
-    size_t status_off = 0, lat_stage_off[2] = {0, 0}, frm_stage_off[2] = {0, 0}, gn_counter_off = 0;
+    size_t status_off = 0, lat_stage_off[2] = {0, 0}, frm_stage_off[2] = {0, 0}, gn_counter_off = 0, stat_off = 0, stat_bytes = 0;
     size_t total = 0;
     // host-transport pipeline (vd_decode_host_stream): two copy streams and the events that order
     // copies and decodes; created on first use, destroyed with the handle
@@ -136,6 +136,24 @@ class Planner {
         gn_toggle_ ^= 1;
         scale_off_ = scale_buf_[gn_toggle_];
         shift_off_ = shift_buf_[gn_toggle_];
+        // On request: where the step before is the tensor-core convolution that writes this very tensor, its epilogue
+        // takes the statistics and the normalisation needs no pass of its own.
+        if ((cfg_.flags & VD_FLAG_FUSED_STATS) && !h_->steps.empty()) {
+            Step& prev = h_->steps.back();
+            ConvArgs probe = prev.conv;
+            probe.B = 1;
+            if (prev.kind == VD_STEP_CONV && prev.use_tc && prev.conv.y == ptr<void>(x_off) && prev.conv.Cout == C &&
+                prev.conv.H == H && prev.conv.W == W && !prev.conv.stat_sum && conv_tc_stats_supported(probe, cfg_.norm_groups)) {
+                ConvArgs& a = prev.conv;
+                a.stat_sum = ptr<unsigned long long>(stat_off_);
+                a.stat_counter = ptr<unsigned int>(stat_off_ + conv_stat_sum_bytes(cfg_.max_batch, cfg_.norm_groups));
+                a.stat_gamma = ptr<float>(g_off); a.stat_beta = ptr<float>(b_off);
+                a.stat_scale = ptr<float>(scale_off_); a.stat_shift = ptr<float>(shift_off_);
+                a.stat_G = cfg_.norm_groups; a.stat_eps = cfg_.norm_eps;
+                prev.info.stats_fused = 1;
+                return;
+            }
+        }
         Step s{};
         s.kind = VD_STEP_GN_STATS;
         s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
@@ -316,6 +334,9 @@ class Planner {
         shift_off_ = shift_buf_[0];
         partial_off_ = alloc(vd_gn_scratch_bytes(B, cfg_.norm_groups));
         h_->gn_counter_off = partial_off_ + gn_partial_bytes(B, cfg_.norm_groups);
+        stat_off_ = alloc(conv_stat_scratch_bytes(B, cfg_.norm_groups));
+        h_->stat_off = stat_off_;
+        h_->stat_bytes = conv_stat_scratch_bytes(B, cfg_.norm_groups);
         zbuf_ = alloc((size_t)B * P0 * lc * 4);
         xs_[0] = alloc((size_t)B * max_x * 4);
         xs_[1] = alloc((size_t)B * max_x * 4);
@@ -391,6 +412,7 @@ class Planner {
     char* base_;
     const vd_config& cfg_;
     size_t cur_ = 0;
+    size_t stat_off_ = 0;
     size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
     size_t scale_buf_[2] = {0, 0}, shift_buf_[2] = {0, 0};
@@ -412,7 +434,7 @@ vd_status validate_cfg(const vd_config* cfg, std::string& err) {
         return VD_ERR_INVALID_ARG;
     }
     if (!(cfg->norm_eps > 0.f) || !(cfg->norm_eps < 1.f)) { err = "norm_eps must be in (0,1)"; return VD_ERR_INVALID_ARG; }
-    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP | VD_FLAG_OUT_U8 | VD_FLAG_CANARY)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
+    if (cfg->flags & ~(VD_FLAG_FORCE_SIMT | VD_FLAG_UPSAMPLE_9TAP | VD_FLAG_OUT_U8 | VD_FLAG_CANARY | VD_FLAG_FUSED_STATS)) { err = "unknown flag bits"; return VD_ERR_INVALID_ARG; }
     return VD_OK;
 }
 
@@ -564,6 +586,7 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
     e = cudaMemsetAsync(h->ws + h->status_off, 0, 256, s);
     // arrival counters of the GroupNorm statistics kernel: zero once, every launch leaves them zero
     if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + h->gn_counter_off, 0, (size_t)cfg->max_batch * 4, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + h->stat_off, 0, h->stat_bytes, s);   // likewise the sums and the counter of the convolutions that take statistics
     for (size_t g : h->guards)
         if (e == cudaSuccess) e = cudaMemsetAsync(h->ws + g, kGuardByte, kGuardBytes, s);
     if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "status memset"); }
@@ -884,6 +907,38 @@ vd_status vd_op_conv2d(const vd_conv_desc* d, const void* x, const void* w_packe
         e = launch_conv_simt(a, (cudaStream_t)cuda_stream);
     }
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_conv2d");
+}
+
+size_t vd_conv_stats_scratch_bytes(int32_t batch, int32_t groups) {
+    if (batch < 1 || groups < 1) return 0;
+    return conv_stat_scratch_bytes(batch, groups);
+}
+
+vd_status vd_op_conv2d_stats(const vd_conv_desc* d, const void* x, const void* w_packed, const float* bias, const float* scale,
+                             const float* shift, void* y, int32_t groups, float eps, const float* gamma, const float* beta,
+                             float* out_scale, float* out_shift, void* scratch, void* cuda_stream) {
+    vd_status st = check_conv_desc(d);
+    if (st != VD_OK) return st;
+    if (!x || !w_packed || !y || !gamma || !beta || !out_scale || !out_shift || !scratch) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
+    if ((scale == nullptr) != (shift == nullptr)) return fail(nullptr, VD_ERR_INVALID_ARG, "scale and shift go together");
+    if (groups < 1) return fail(nullptr, VD_ERR_INVALID_ARG, "bad group count");
+    if (d->batch == 0) return VD_OK;
+    ConvArgs a = conv_args_from_desc(d);
+    a.x = x; a.w = w_packed; a.bias = bias; a.scale = scale; a.shift = shift; a.y = y;
+    bool tc;
+    st = resolve_impl(d, a, &tc);
+    if (st != VD_OK) return st;
+    if (!tc || !conv_tc_stats_supported(a, groups))
+        return fail(nullptr, VD_ERR_UNSUPPORTED, "this layer's epilogue cannot take GroupNorm statistics");
+    a.stat_sum = (unsigned long long*)scratch;
+    a.stat_counter = (unsigned int*)((char*)scratch + conv_stat_sum_bytes(a.B, groups));
+    a.stat_gamma = gamma; a.stat_beta = beta; a.stat_scale = out_scale; a.stat_shift = out_shift;
+    a.stat_G = groups; a.stat_eps = eps;
+    cudaError_t e = cudaMemsetAsync(scratch, 0, conv_stat_scratch_bytes(a.B, groups), (cudaStream_t)cuda_stream);
+    ConvTcPlan plan{};
+    if (e == cudaSuccess) e = conv_tc_prepare(a, &plan);
+    if (e == cudaSuccess) e = launch_conv_tc(a, plan, nullptr, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_conv2d_stats");
 }
 
 size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups) {

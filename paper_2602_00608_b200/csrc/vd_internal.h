@@ -32,11 +32,25 @@ struct ConvArgs {
     const void* w2;         // fp32 [Cout][Cin2] (tensor-core kernel: the shortcut's products are tf32)
     const float* bias2;     // [Cout] or null
     int Cin2;
+    // optional (tensor-core kernel only): the GroupNorm that follows takes its statistics from this layer's
+    // epilogue instead of a pass of its own.  Every epilogue warp adds (sum, sum of squares) of the output it
+    // drained, in 64-bit fixed point, per group; the CTA that finishes last turns the sums into scale and shift.
+    unsigned long long* stat_sum;   // [B][stat_G][2] sums, or null; zero before the launch, left zero
+    unsigned int* stat_counter;  // CTAs done; zero before the launch, left zero
+    const float* stat_gamma;     // [Cout]
+    const float* stat_beta;      // [Cout]
+    float* stat_scale;           // [B,Cout]
+    float* stat_shift;           // [B,Cout]
+    int stat_G;
+    float stat_eps;
     // tensor-core kernel: ceil(2^32 / d) for the divisors of its tile numbering (tiles per image, channel
     // blocks, tiles per row), filled in by its launcher; 0 stands for d = 1
     unsigned int div_tiles, div_nblk, div_tx;
 };
 constexpr int kConvMaxCtas = 160;         // upper bound on the persistent grid
+// bytes of the statistics sums of a convolution's epilogue, then its arrival counter
+inline size_t conv_stat_sum_bytes(int B, int G) { return (((size_t)B * G * 2 * sizeof(unsigned long long)) + 255) / 256 * 256; }
+inline size_t conv_stat_scratch_bytes(int B, int G) { return conv_stat_sum_bytes(B, G) + 256; }
 
 struct GnArgs {
     const void* x;          // NHWC [B,H,W,C]
@@ -94,6 +108,7 @@ cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cud
 
 // ---- tcgen05 kernels (conv_tc.cu, attn_tc.cu)
 bool conv_tc_supported(const ConvArgs& a);
+bool conv_tc_stats_supported(const ConvArgs& a, int groups);   // the epilogue can take the next GroupNorm's statistics
 bool conv_tc_pairs_available();          // can the current device co-schedule the kernels' CTA pairs?
 size_t conv_tc_packed_bytes(int Cout, int Cin, int taps, bool phase);
 // OIHW weight (bf16) -> bf16 [tap][Cout_pad][Cin] (K-major rows for the B operand); phase: the sixteen

@@ -37,7 +37,7 @@ def test_struct_sizes_match_the_header_layout(vd):
     assert ctypes.sizeof(vd.VdConfig) == 44
     assert ctypes.sizeof(vd.VdTensor) == 56
     assert ctypes.sizeof(vd.VdConvDesc) == 56
-    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 16
+    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 24
 
 
 def test_query_workspace_is_host_only_and_scales_with_batch(vd):

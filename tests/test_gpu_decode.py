@@ -71,9 +71,10 @@ def test_sdvae_fp32_path_matches_oracle(env):
     assert rel_l2(got.cpu().numpy(), want) <= F32_REL_L2
 
 
-@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1, 0x10])
 def test_sdvae_bf16_ragged_tiles_batch2(env, flags):
     # 20x28 latents: every level's width/height leaves a ragged last tile; two frames
+    # (flags: default, FFMA kernels, GroupNorm statistics taken in the convolutions' epilogues)
     torch, ref, vd, synth = env
     wl = synth.WORKLOADS[3]
     z = synth.workload_latents(wl, batch=2, h=20, w=28)
@@ -167,6 +168,27 @@ def test_sdvae_bf16_degenerate_and_odd_sizes(env, h, w, b):
         g = got.float().cpu().numpy()
         assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
     dec.check_status()
+
+
+def test_fused_statistics_replace_the_norm2_passes(env):
+    """VD_FLAG_FUSED_STATS: the second GroupNorm of every ResNet block has no step of its own (its statistics come
+    from conv1's epilogue), and the frame stays within the bf16 bound of the default path's frame
+    (the oracle comparison of this mode is test_sdvae_bf16_ragged_tiles_batch2[16])."""
+    torch, ref, vd, synth = env
+    wl = synth.WORKLOADS[2]
+    z = synth.workload_latents(wl, batch=1, h=12, w=20)
+    dec, got, _ = _decode(env, wl, z)
+    dec2, got2, _ = _decode(env, wl, z, flags=vd.VD_FLAG_FUSED_STATS)
+    s1, s2 = dec.steps(), dec2.steps()
+    gn1 = [s["name"] for s in s1 if s["kind"] == vd.VD_STEP_GN_STATS]
+    gn2 = [s["name"] for s in s2 if s["kind"] == vd.VD_STEP_GN_STATS]
+    fused = [s["name"] for s in s2 if s.get("stats_fused")]
+    assert len(fused) > 0 and len(gn1) - len(gn2) == len(fused)
+    assert all(n.endswith("conv1") for n in fused) and not any(n.endswith("norm2") for n in gn2)
+    assert not any(s.get("stats_fused") for s in s1)
+    d = got.float() - got2.float()
+    assert float(d.norm() / got.float().norm()) <= BF16_REL_L2      # (bf16 roundings flip between two correct paths)
+    dec2.check_status()
 
 
 def test_platformer_shape_256x256_stream_against_the_oracle(env):

@@ -309,6 +309,67 @@ def test_conv_tc_matches_oracle(env, case):
     assert rel_l2(got, got2) <= (4e-3 if case["out_bf16"] else (2e-4 if case["silu"] else 2e-5))
 
 
+STAT_CASES = [
+    # B, H, W, Cin, Cout, k, G, prologue  (channels per group 4, 8, 16; one- and two-tile items, CTA pairs, ragged edges)
+    (1, 16, 8, 64, 128, 3, 32, False),
+    (2, 19, 13, 64, 128, 3, 32, False),
+    (1, 37, 29, 128, 256, 3, 32, False),
+    (3, 9, 21, 64, 512, 3, 32, False),
+    (1, 60, 90, 64, 512, 1, 32, False),
+    (2, 33, 17, 64, 128, 3, 8, False),
+    (1, 23, 31, 128, 256, 3, 32, True),
+]
+
+
+@pytest.mark.parametrize("B,H,W,Cin,Cout,k,G,prologue", STAT_CASES)
+def test_conv_tc_epilogue_statistics_match_oracle(env, B, H, W, Cin, Cout, k, G, prologue):
+    """The GroupNorm statistics a convolution's epilogue takes of its own output against the oracle's two-pass
+    statistics of the oracle's convolution.  Without a prologue the bf16 operands are exact on both sides, so the
+    values differ by fp32 accumulation only and the bound is tight."""
+    torch, ref, vd, synth = env
+    r = _rng(77 + Cout + H)
+    x = synth.round_to_bf16(r.standard_normal((B, Cin, H, W)).astype(np.float32) * 1.5 + 0.3)
+    w = synth.round_to_bf16((r.uniform(-1, 1, (Cout, Cin, k, k)) * math.sqrt(3.0 / (Cin * k * k))).astype(np.float32))
+    bias = r.uniform(-0.5, 0.5, Cout).astype(np.float32)
+    gamma = r.uniform(0.9, 1.1, Cout).astype(np.float32)
+    beta = r.uniform(-0.1, 0.1, Cout).astype(np.float32)
+    scale = r.uniform(0.5, 1.5, (B, Cin)).astype(np.float32) if prologue else None
+    shift = r.uniform(-0.5, 0.5, (B, Cin)).astype(np.float32) if prologue else None
+    t = x
+    if prologue:
+        t = ref.silu(t * scale[:, :, None, None] + shift[:, :, None, None])
+    want = ref.conv2d(t, w, bias)
+    _, mean, rstd = ref.groupnorm(want, gamma, beta, G, 1e-6, return_stats=True)
+    cpg = Cout // G
+    want_scale = gamma[None, :] * np.repeat(rstd, cpg, axis=1)
+    want_shift = beta[None, :] - np.repeat(mean, cpg, axis=1) * want_scale
+    dev = lambda a: None if a is None else torch.from_numpy(a).cuda()
+    y, sc, sh = vd.op_conv2d_stats(util.nchw_to_dev_nhwc(x, torch.bfloat16), torch.from_numpy(w).cuda().to(torch.bfloat16),
+                                   dev(gamma), dev(beta), G, 1e-6, dev(bias), dev(scale), dev(shift), silu=prologue)
+    y2, sc2, sh2 = vd.op_conv2d_stats(util.nchw_to_dev_nhwc(x, torch.bfloat16), torch.from_numpy(w).cuda().to(torch.bfloat16),
+                                      dev(gamma), dev(beta), G, 1e-6, dev(bias), dev(scale), dev(shift), silu=prologue)
+    torch.cuda.synchronize()
+    got = util.dev_nhwc_to_nchw(y)
+    assert rel_l2(got, want) <= 1e-2
+    tol = 3e-3 if prologue else 1e-4
+    np.testing.assert_allclose(sc.cpu().numpy(), want_scale, rtol=tol)
+    np.testing.assert_allclose(sh.cpu().numpy(), want_shift, rtol=tol, atol=tol)
+    assert torch.equal(sc, sc2) and torch.equal(sh, sh2) and torch.equal(y, y2)      # fixed summation order
+
+
+def test_conv_tc_epilogue_statistics_unsupported_layers_say_so(env):
+    torch, ref, vd, synth = env
+    x = torch.zeros((1, 8, 8, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((128, 64, 3, 3), dtype=torch.bfloat16, device="cuda")
+    g = torch.ones(128, device="cuda")
+    with pytest.raises(vd.VdError) as e:
+        vd.op_conv2d_stats(x, w, g, g, 64, 1e-6)          # two channels per group
+    assert e.value.status == vd.VD_ERR_UNSUPPORTED
+    with pytest.raises(vd.VdError) as e:
+        vd.op_conv2d_stats(x, w, g, g, 32, 1e-6, impl=vd.VD_IMPL_SIMT)
+    assert e.value.status == vd.VD_ERR_UNSUPPORTED
+
+
 def test_conv_tc_real_layer_shape_sampled(env):
     """A full-size layer (128->128 at 480x720, the most common launch of the headline workload):
     sampled windows of the output against the oracle run on crops of the same seeded input."""
