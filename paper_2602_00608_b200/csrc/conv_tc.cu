@@ -91,7 +91,7 @@ constexpr int WARP_SLICE_BYTES = 32 * 128;                           // one epil
 // accumulator's last MMA and its next first MMA lie the MMAs of six (parity, chunk) blocks.  An operand
 // chunk therefore stays in shared memory for four slots (five stages).  PhaseSched is that schedule; the
 // weight loader follows it step by step.
-template <int BN, int CG = 1, bool PH = false> struct TileCfg {
+template <int BN, int CG = 1, bool PH = false, bool IN_BF16 = false> struct TileCfg {
     static_assert(CG == 1 || BN >= 128, "the two-CTA form exists for 128- and 256-channel blocks");
     static_assert(!PH || (BN == 128 && CG == 2), "the phase form runs 128-channel blocks on CTA pairs");
     static constexpr int PAIR = PH ? 1 : (BN == 256 ? 1 : 2);        // tiles per work item (and CTA)
@@ -99,7 +99,9 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     // output slices per epilogue warp (128-channel blocks: a second slice buffer pays more than a fourth weight stage)
     static constexpr int OUT_BUFS = (PH || BN == 128) ? 2 : 1;
     // weight stages: as many as fit (the weight stream waits on the latency of L2, which the SM clock does not shorten)
-    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? 3 : 8)));
+    // (128-channel blocks: the staging of a bf16 input is half the size, which buys a fourth stage; measured, the MMA
+    // warp of such a layer waits on weights for a quarter of its time with three)
+    static constexpr int B_STAGES = PH ? 4 : (CG == 2 ? (BN == 256 ? 7 : 8) : (BN == 256 ? 5 : (BN == 128 ? (IN_BF16 ? 4 : 3) : 8)));
     static constexpr int B_GROUP = BN >= 128 ? 1 : 2;                // weight stages handed back per tcgen05.commit
     static constexpr int A_STAGES = PH ? 5 : 2;                    // phase form: a chunk stays until the parity that lags most has used it
     static constexpr int A_STAGE_BYTES = PAIR * A_TILE_BYTES;
@@ -110,7 +112,7 @@ template <int BN, int CG = 1, bool PH = false> struct TileCfg {
     static constexpr int SMEM_BARS = 512;
     // two-tile items and two-CTA pairs: the producers stage the raw input of the next unit in shared memory (cp.async)
     static constexpr bool STAGED = !PH && (PAIR == 2 || CG == 2);
-    static constexpr int SMEM_RAW = STAGED ? ITEMS * 32 : 0;
+    static constexpr int SMEM_RAW = STAGED ? ITEMS * (IN_BF16 ? 16 : 32) : 0;
     static constexpr int SMEM_TOTAL = SMEM_B + SMEM_OUT + SMEM_A + SMEM_BIAS + SMEM_BARS + SMEM_RAW + 1024;  // + barriers + alignment slack
     static constexpr int ACC_COLS = BN < 32 ? 32 : BN;               // TMEM columns per accumulator
     static constexpr int NBUF = PH ? 1 : 2;                          // accumulator sets (PAIR tiles each; phase: four parities)
@@ -335,7 +337,7 @@ template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
-    using Cfg = TileCfg<BN, CG, PH>;
+    using Cfg = TileCfg<BN, CG, PH, IN_BF16>;
     constexpr int NBUF = Cfg::NBUF, PAIR = Cfg::PAIR, A_STAGE_BYTES = Cfg::A_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -1420,7 +1422,7 @@ cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, 
 template <int BN, bool IB, int OM, int CG, bool PH = false>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
     auto kern = conv_tc_kernel<BN, IB, OM, CG, PH>;
-    constexpr int SMEM = TileCfg<BN, CG, PH>::SMEM_TOTAL;
+    constexpr int SMEM = TileCfg<BN, CG, PH, IB>::SMEM_TOTAL;
     static KernelState state = {};
     int pairs = 0, sms = 0;
     cudaError_t e = kernel_state(kern, SMEM, CG, state, &pairs, &sms);
