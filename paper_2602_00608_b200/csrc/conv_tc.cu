@@ -333,7 +333,9 @@ __device__ void stat_finalize(const ConvArgs& a, int tid, void* smem_scratch) {
 
 // OUT_MODE: 0 = fp32 NHWC, 1 = bf16 NHWC (both through shared memory and TMA stores),
 //           2 = NCHW frame written directly (dtype from a.out_dtype)
-template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false>
+// STATS: the epilogue also takes the GroupNorm statistics of the output (a build of its own: compiled in but switched
+// off, the extra live values cost the bf16-output kernels 1.4 % of a decode in spills)
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
@@ -788,7 +790,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const uint64_t pol_out = l2_policy_evict_last();
             // statistics for the normalisation that follows: per-pass totals of the current (frame, channel block) run
             constexpr int NPS = NP > 0 ? NP : 1;
-            const bool stats = OUT_MODE == 1 && !PH && NP > 0 && a.stat_sum != nullptr;
+            constexpr bool stats = STATS && OUT_MODE == 1 && !PH && NP > 0;
             long long sacc[NPS];
 #pragma unroll
             for (int p = 0; p < NPS; ++p) sacc[p] = 0;
@@ -1276,7 +1278,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
         if (CG == 2) tmem_dealloc2(tmem_base, (uint32_t)Cfg::TMEM_COLS);
         else tmem_dealloc(tmem_base, (uint32_t)Cfg::TMEM_COLS);
     }
-    if (OUT_MODE != 2 && a.stat_sum) {
+    if (STATS && OUT_MODE == 1) {
         // every sum of this CTA has been added (and fenced) before the barrier above
         if (tid == 0) {
             __threadfence();
@@ -1419,9 +1421,9 @@ cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, 
     return cudaSuccess;
 }
 
-template <int BN, bool IB, int OM, int CG, bool PH = false>
+template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH>;
+    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS>;
     constexpr int SMEM = TileCfg<BN, CG, PH, IB>::SMEM_TOTAL;
     static KernelState state = {};
     int pairs = 0, sms = 0;
@@ -1635,6 +1637,11 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
     }
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
+    }
+    if (a.stat_sum) {          // bf16 output with the statistics of the following GroupNorm (checked above)
+        if (plan.bn == 256 && plan.cg == 2) return ib ? launch_one<256, true, 1, 2, false, true>(a, plan, status, s) : launch_one<256, false, 1, 2, false, true>(a, plan, status, s);
+        if (plan.bn == 256) return ib ? launch_one<256, true, 1, 1, false, true>(a, plan, status, s) : launch_one<256, false, 1, 1, false, true>(a, plan, status, s);
+        return ib ? launch_one<128, true, 1, 1, false, true>(a, plan, status, s) : launch_one<128, false, 1, 1, false, true>(a, plan, status, s);
     }
     if (plan.bn == 256 && plan.cg == 2) {
         if (ib && ob) return launch_one<256, true, 1, 2>(a, plan, status, s);
