@@ -48,6 +48,9 @@ typedef struct {
     int32_t stats_fused;        /* 1: a convolution whose epilogue also produces the statistics (scale, shift) of the
                                    GroupNorm that follows; that GroupNorm has no step of its own then */
     int32_t reserved;
+    int64_t out_pending_offset; /* >= 0: byte offset in the workspace of an fp32 vector [out_channels]; the step's stored
+                                   output lacks this per-channel constant (a bias left out of the epilogue and accounted
+                                   for by the steps that read the tensor): layer output = stored + pending[c].  -1: none */
 } vd_step_info;
 
 VD_API vd_status vd_num_steps(vd_handle h, int32_t* n);
@@ -133,13 +136,15 @@ VD_API vd_status vd_op_conv2d_stats(const vd_conv_desc* d, const void* x, const 
 
 /* GroupNorm statistics of x (device NHWC [batch,h,w,c], dtype `dtype`) folded with the affine
  * parameters: scale[n,c] = gamma[c]*rstd[n,g], shift[n,c] = beta[c] - mean[n,g]*scale[n,c]
- * (biased variance, eps inside the root).  `scratch` is device memory of
+ * (biased variance, eps inside the root).  `offset` (device fp32 [c], or NULL): the statistics are those
+ * of x[..,c] + offset[c] and shift takes scale*offset in, so that scale*x + shift is GroupNorm(x + offset):
+ * the decoder leaves a convolution's bias out of its epilogue and lets the next normalisation account for it.  `scratch` is device memory of
  * vd_gn_scratch_bytes(batch, groups) bytes (chunk records, then one arrival counter per sample,
  * which the call clears itself).  scale/shift are device fp32 [batch,c].  c <= 1024, c/groups a
  * multiple of 4.  One kernel launch; results are bitwise reproducible and do not depend on batch. */
 VD_API size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups);
 VD_API vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w, int32_t c,
-                                int32_t groups, float eps, const float* gamma, const float* beta,
+                                int32_t groups, float eps, const float* gamma, const float* beta, const float* offset,
                                 float* scale, float* shift, void* scratch, void* cuda_stream);
 
 /* The same operator for callers that cannot hand over (or allocate) a scratch buffer.  The paper

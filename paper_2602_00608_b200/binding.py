@@ -49,7 +49,7 @@ class VdStepInfo(Structure):
                 ("out_nchw", c_int32), ("out_offset", c_int64), ("flops_per_frame", c_double),
                 ("bytes_per_frame", c_double), ("weight_bytes", c_double), ("c_in2", c_int32),
                 ("has_residual", c_int32), ("phase_collapsed", c_int32), ("out_u8", c_int32),
-                ("stats_fused", c_int32), ("reserved", c_int32)]
+                ("stats_fused", c_int32), ("reserved", c_int32), ("out_pending_offset", c_int64)]
 
 
 class VdConvDesc(Structure):
@@ -102,7 +102,7 @@ def lib():
         l.vd_op_conv2d_stats.argtypes = [POINTER(VdConvDesc), vp, vp, vp, vp, vp, vp, c_int32, c_float, vp, vp, vp, vp, vp, vp]
         l.vd_gn_scratch_bytes.argtypes = [c_int32, c_int32]
         l.vd_gn_scratch_bytes.restype = c_size_t
-        l.vd_op_gn_stats.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp, vp]
+        l.vd_op_gn_stats.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp, vp, vp]
         l.vd_op_gn_stats_static.argtypes = [vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, vp, vp, vp, vp, vp]
         l.vd_op_attention.argtypes = [vp, vp, vp, vp, c_int32, c_int32, c_int32, c_int32, c_int32, c_int32, c_float, c_int32, vp, vp]
         l.vd_attention_scratch_bytes.argtypes = [c_int32, c_int32, c_int32]
@@ -274,14 +274,19 @@ class Decoder:
         _check(lib().vd_debug_stop_after(self.handle, index), self.handle)
 
     def read_step_output(self, step: dict, batch: int):
-        """The output tensor of a step, from the workspace, as an fp32 NCHW torch tensor (device)."""
+        """The output of a step as an fp32 NCHW torch tensor (device): the stored tensor from the workspace plus,
+        where the step left its bias pending (out_pending_offset), that per-channel vector."""
         torch = self.torch
         dt = _torch_dtype(step["out_dtype"])
-        n = batch * step["out_h"] * step["out_w"] * step["out_channels"]
+        c = step["out_channels"]
+        n = batch * step["out_h"] * step["out_w"] * c
         es = 2 if step["out_dtype"] == VD_BF16 else 4
         raw = self.workspace[step["out_offset"]: step["out_offset"] + n * es].view(dt)
-        t = raw.view(batch, step["out_h"], step["out_w"], step["out_channels"])
-        return t.permute(0, 3, 1, 2).float().contiguous()
+        t = raw.view(batch, step["out_h"], step["out_w"], c).float()
+        po = step.get("out_pending_offset", -1)
+        if po >= 0:
+            t = t + self.workspace[po: po + 4 * c].view(torch.float32)
+        return t.permute(0, 3, 1, 2).contiguous()
 
     def close(self):
         if getattr(self, "handle", None):
@@ -356,15 +361,15 @@ def op_conv2d_stats(x_nhwc, w_oihw, gamma, beta, groups: int, eps: float, bias=N
     return y, out_scale, out_shift
 
 
-def op_gn_stats(x_nhwc, gamma, beta, groups: int, eps: float):
-    """Per-(sample, channel) GroupNorm scale and shift of an NHWC device tensor."""
+def op_gn_stats(x_nhwc, gamma, beta, groups: int, eps: float, offset=None):
+    """Per-(sample, channel) GroupNorm scale and shift of an NHWC device tensor (of x + offset[c] if given)."""
     import torch
     b, h, w, c = x_nhwc.shape
     scratch = torch.empty(max(1, lib().vd_gn_scratch_bytes(max(b, 1), groups)), dtype=torch.uint8, device=x_nhwc.device)
     scale = torch.empty((b, c), dtype=torch.float32, device=x_nhwc.device)
     shift = torch.empty((b, c), dtype=torch.float32, device=x_nhwc.device)
-    p = lambda t: c_void_p(t.data_ptr())
-    _check(lib().vd_op_gn_stats(p(x_nhwc.contiguous()), _dt(x_nhwc), b, h, w, c, groups, eps, p(gamma), p(beta), p(scale), p(shift), p(scratch), _stream_ptr()))
+    p = lambda t: None if t is None else c_void_p(t.data_ptr())
+    _check(lib().vd_op_gn_stats(p(x_nhwc.contiguous()), _dt(x_nhwc), b, h, w, c, groups, eps, p(gamma), p(beta), p(offset), p(scale), p(shift), p(scratch), _stream_ptr()))
     return scale, shift
 
 

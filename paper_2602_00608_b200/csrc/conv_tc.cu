@@ -335,7 +335,9 @@ __device__ void stat_finalize(const ConvArgs& a, int tid, void* smem_scratch) {
 //           2 = NCHW frame written directly (dtype from a.out_dtype)
 // STATS: the epilogue also takes the GroupNorm statistics of the output (a build of its own: compiled in but switched
 // off, the extra live values cost the bf16-output kernels 1.4 % of a decode in spills)
-template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false>
+// BIAS: the epilogue adds the bias (a build without it for the layers whose bias is accounted for downstream: the
+// additions and the bias loads are more than half of a pass's instructions)
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false, bool BIAS = true>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
@@ -786,6 +788,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             // critical path (two accumulator sets), and the shared memory saved is one more weight stage.
             uint8_t* wout = smem_out + ew * (Cfg::OUT_BUFS * WARP_SLICE_BYTES);
             float* wbias = (float*)(smem_bias) + ew * BN;                    // this warp's copy of the block's bias
+            constexpr bool has_bias = BIAS || OUT_MODE == 2;
             int bias_n0 = -1;
             const uint64_t pol_out = l2_policy_evict_last();
             // statistics for the normalisation that follows: per-pass totals of the current (frame, channel block) run
@@ -837,7 +840,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const int m = ew * 32 + lane;
                         stat_valid = tl.ty0 + (m >> 3) < a.H && tl.tx0 + (m & 7) < a.W;
                     }
-                    if (tl.n0 != bias_n0) {                   // (re)load bias (+ shortcut bias) of this channel block
+                    if (has_bias && tl.n0 != bias_n0) {       // (re)load bias (+ shortcut bias) of this channel block
                         __syncwarp();
                         for (int i = lane; i < BN; i += 32)
                             wbias[i] = (a.bias ? __ldg(a.bias + tl.n0 + i) : 0.f) + (a.bias2 ? __ldg(a.bias2 + tl.n0 + i) : 0.f);
@@ -876,13 +879,27 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         uint8_t* orow = obuf + lane * 128;
                         const float4* bp = (const float4*)(wbias + p * 32);
                         if (OUT_MODE == 0) {
+                            if (has_bias) {
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) {
-                                const float4 tb = bp[c];
-                                *(float4*)(orow + ((c ^ (lane & 7)) << 4)) =
-                                    make_float4(__uint_as_float(rc[4 * c]) + tb.x, __uint_as_float(rc[4 * c + 1]) + tb.y,
-                                                __uint_as_float(rc[4 * c + 2]) + tb.z, __uint_as_float(rc[4 * c + 3]) + tb.w);
+                                for (int c = 0; c < 8; ++c) {
+                                    const float4 tb = bp[c];
+                                    *(float4*)(orow + ((c ^ (lane & 7)) << 4)) =
+                                        make_float4(__uint_as_float(rc[4 * c]) + tb.x, __uint_as_float(rc[4 * c + 1]) + tb.y,
+                                                    __uint_as_float(rc[4 * c + 2]) + tb.z, __uint_as_float(rc[4 * c + 3]) + tb.w);
+                                }
+                            } else {                              // the accumulator as it is (the bias is accounted for downstream)
+#pragma unroll
+                                for (int c = 0; c < 8; ++c)
+                                    *(uint4*)(orow + ((c ^ (lane & 7)) << 4)) = make_uint4(rc[4 * c], rc[4 * c + 1], rc[4 * c + 2], rc[4 * c + 3]);
                             }
+                        } else if (!stats && !has_bias) {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                *(uint4*)(orow + (((h * 4 + c) ^ (lane & 7)) << 4)) =
+                                    make_uint4(pack_bf16(__uint_as_float(rc[8 * c]), __uint_as_float(rc[8 * c + 1])),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 2]), __uint_as_float(rc[8 * c + 3])),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 4]), __uint_as_float(rc[8 * c + 5])),
+                                               pack_bf16(__uint_as_float(rc[8 * c + 6]), __uint_as_float(rc[8 * c + 7])));
                         } else {
                             float v[8];
                             const bool stat_hi = (lane & 16) != 0;
@@ -1421,9 +1438,9 @@ cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, 
     return cudaSuccess;
 }
 
-template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false>
+template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false, bool BIAS = true>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS>;
+    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS, BIAS>;
     constexpr int SMEM = TileCfg<BN, CG, PH, IB>::SMEM_TOTAL;
     static KernelState state = {};
     int pairs = 0, sms = 0;
@@ -1629,36 +1646,27 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
     if (a.stat_sum && (!conv_tc_stats_supported(a, a.stat_G) || !a.stat_counter || !a.stat_scale || !a.stat_shift || !a.stat_gamma || !a.stat_beta))
         return cudaErrorInvalidValue;
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
-    if (plan.phase) {
-        if (ib && ob) return launch_one<128, true, 1, 2, true>(a, plan, status, s);
-        if (ib && !ob) return launch_one<128, true, 0, 2, true>(a, plan, status, s);
-        if (!ib && ob) return launch_one<128, false, 1, 2, true>(a, plan, status, s);
-        return launch_one<128, false, 0, 2, true>(a, plan, status, s);
-    }
-    if (plan.bn == 16) {
-        return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
-    }
+    const bool hb = a.bias != nullptr || a.bias2 != nullptr;
     if (a.stat_sum) {          // bf16 output with the statistics of the following GroupNorm (checked above)
         if (plan.bn == 256 && plan.cg == 2) return ib ? launch_one<256, true, 1, 2, false, true>(a, plan, status, s) : launch_one<256, false, 1, 2, false, true>(a, plan, status, s);
         if (plan.bn == 256) return ib ? launch_one<256, true, 1, 1, false, true>(a, plan, status, s) : launch_one<256, false, 1, 1, false, true>(a, plan, status, s);
         return ib ? launch_one<128, true, 1, 1, false, true>(a, plan, status, s) : launch_one<128, false, 1, 1, false, true>(a, plan, status, s);
     }
-    if (plan.bn == 256 && plan.cg == 2) {
-        if (ib && ob) return launch_one<256, true, 1, 2>(a, plan, status, s);
-        if (ib && !ob) return launch_one<256, true, 0, 2>(a, plan, status, s);
-        if (!ib && ob) return launch_one<256, false, 1, 2>(a, plan, status, s);
-        return launch_one<256, false, 0, 2>(a, plan, status, s);
+    if (plan.bn == 16) {
+        return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
     }
-    if (plan.bn == 256) {
-        if (ib && ob) return launch_one<256, true, 1, 1>(a, plan, status, s);
-        if (ib && !ob) return launch_one<256, true, 0, 1>(a, plan, status, s);
-        if (!ib && ob) return launch_one<256, false, 1, 1>(a, plan, status, s);
-        return launch_one<256, false, 0, 1>(a, plan, status, s);
-    }
-    if (ib && ob) return launch_one<128, true, 1, 1>(a, plan, status, s);
-    if (ib && !ob) return launch_one<128, true, 0, 1>(a, plan, status, s);
-    if (!ib && ob) return launch_one<128, false, 1, 1>(a, plan, status, s);
-    return launch_one<128, false, 0, 1>(a, plan, status, s);
+#define VD_CONV_CASE(BN_, CG_, PH_)                                                                                         \
+    do {                                                                                                                    \
+        if (ib && ob) return hb ? launch_one<BN_, true, 1, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, true, 1, CG_, PH_, false, false>(a, plan, status, s);     \
+        if (ib && !ob) return hb ? launch_one<BN_, true, 0, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, true, 0, CG_, PH_, false, false>(a, plan, status, s);    \
+        if (!ib && ob) return hb ? launch_one<BN_, false, 1, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, false, 1, CG_, PH_, false, false>(a, plan, status, s);  \
+        return hb ? launch_one<BN_, false, 0, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, false, 0, CG_, PH_, false, false>(a, plan, status, s);                 \
+    } while (0)
+    if (plan.phase) VD_CONV_CASE(128, 2, true);
+    if (plan.bn == 256 && plan.cg == 2) VD_CONV_CASE(256, 2, false);
+    if (plan.bn == 256) VD_CONV_CASE(256, 1, false);
+    VD_CONV_CASE(128, 1, false);
+#undef VD_CONV_CASE
 }
 
 }  // namespace vd

@@ -102,23 +102,39 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
     __shared__ float2 sm[kGnThreads];
     __shared__ int s_last;
     griddep_launch();
+    const int slots = a.C / 4;                       // 4-channel slots per pixel (<= kGnThreads)
+    const int cpg = a.C / a.G;
+    const int slot = threadIdx.x % slots;
+    // The per-channel offset does not depend on the kernel before this one: it is read while that kernel finishes.
+    // off_k: what the offset adds to the group's reference value; off_c: this thread's four channels;
+    // off_fin: the same reference term for the group this thread finalises (threads below G, last block only).
+    float off_k = 0.f, off_fin = 0.f;
+    float4 off_c = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (a.offset) {
+        const float4 og = __ldg((const float4*)(a.offset + (slot * 4 / cpg) * cpg));
+        off_k = 0.25f * ((og.x + og.y) + (og.z + og.w));
+        off_c = __ldg((const float4*)(a.offset + slot * 4));
+        if (threadIdx.x < a.G) {
+            const float4 of = __ldg((const float4*)(a.offset + threadIdx.x * cpg));
+            off_fin = 0.25f * ((of.x + of.y) + (of.z + of.w));
+        }
+    }
     griddep_wait();
     const int n = blockIdx.y;
     const int chunk = blockIdx.x;
-    const int slots = a.C / 4;                       // 4-channel slots per pixel (<= kGnThreads)
     const int p0 = chunk * pix_per_chunk;
     const int p1 = min(a.P, p0 + pix_per_chunk);
     const T* x = (const T*)a.x + (size_t)n * a.P * a.C;
-    const int cpg = a.C / a.G;
     const int rows = kGnThreads / slots;             // pixels handled side by side
-    const int slot = threadIdx.x % slots;
     const int row = threadIdx.x / slots;
 
     float s = 0.f, ss = 0.f;
     if (row < rows && p0 + row < p1) {
         float kv[4];
         load4<T>(x + (size_t)(a.P / 2) * a.C + (slot * 4 / cpg) * cpg, kv);
-        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
+        // a per-channel offset is taken into the reference value: d = (x + off) - k = x - (k - off)
+        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3])) + off_k;
+        const float ko[4] = {k - off_c.x, k - off_c.y, k - off_c.z, k - off_c.w};
         int p = p0 + row;
         const uint64_t pol = policy_evict_first();
         for (; p + (U - 1) * rows < p1; p += U * rows) {        // U independent loads in flight
@@ -129,7 +145,7 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
             for (int j = 0; j < U; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float d = u[j][e] - k;
+                    const float d = u[j][e] - ko[e];
                     s += d;
                     ss = fmaf(d, d, ss);
                 }
@@ -139,7 +155,7 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
             load4<T>(x + (size_t)p * a.C + slot * 4, v);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float d = v[e] - k;
+                const float d = v[e] - ko[e];
                 s += d;
                 ss = fmaf(d, d, ss);
             }
@@ -210,7 +226,7 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
         }
         float kv[4];
         load4<T>(x + (size_t)(a.P / 2) * a.C + threadIdx.x * cpg, kv);
-        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3]));
+        const float k = 0.25f * ((kv[0] + kv[1]) + (kv[2] + kv[3])) + off_fin;
         const float inv_n = 1.f / ((float)a.P * (float)cpg);
         const float md = t.x * inv_n;
         const float var = fmaxf(fmaf(-md, md, t.y * inv_n), 0.f);
@@ -222,7 +238,7 @@ __global__ void __launch_bounds__(kGnThreads, 2) gn_stats_kernel(GnArgs a, int c
         const int gc = c / cpg;
         const float sc = __ldg(a.gamma + c) * s_rstd[gc];
         a.scale[(size_t)n * a.C + c] = sc;
-        a.shift[(size_t)n * a.C + c] = __ldg(a.beta + c) - s_mean[gc] * sc;
+        a.shift[(size_t)n * a.C + c] = __ldg(a.beta + c) - (s_mean[gc] - (a.offset ? __ldg(a.offset + c) : 0.f)) * sc;
     }
     if (threadIdx.x == 0) a.counters[n] = 0u;        // ready for the next launch
 }
@@ -556,6 +572,33 @@ cudaError_t launch_pack_weight_simt(const void* w, int w_dtype, float* packed, i
     return cudaGetLastError();
 }
 
+__global__ void fold_bias_kernel(float* out, const float* in, const float* b, const float* b2, const float* w2, const float* pin,
+                                 int Cin2, int Cout) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= Cout) return;
+    float v = (in ? in[c] : 0.f) + (b ? b[c] : 0.f) + (b2 ? b2[c] : 0.f);
+    if (w2 && pin) {
+        float acc = 0.f;
+        for (int k = 0; k < Cin2; ++k) acc = fmaf(w2[(size_t)c * Cin2 + k], pin[k], acc);
+        v += acc;
+    }
+    out[c] = v;
+}
+__global__ void fill_rows_kernel(float* dst, const float* src, int C, int B) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < C * B) dst[i] = src ? src[i % C] : 1.f;
+}
+cudaError_t launch_fold_bias(float* out, const float* in, const float* b, const float* b2, const float* w2, const float* pin,
+                             int Cin2, int Cout, cudaStream_t s) {
+    fold_bias_kernel<<<(Cout + 127) / 128, 128, 0, s>>>(out, in, b, b2, w2, pin, Cin2, Cout);
+    return cudaGetLastError();
+}
+cudaError_t launch_fill_rows(float* dst, const float* src, int C, int B, cudaStream_t s) {
+    const int n = C * B;
+    fill_rows_kernel<<<(n + 255) / 256, 256, 0, s>>>(dst, src, C, B);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cudaStream_t s) {
     if (dtype == VD_BF16) to_f32_kernel<__nv_bfloat16><<<grid_for(n, 256), 256, 0, s>>>((const __nv_bfloat16*)src, dst, n);
     else to_f32_kernel<float><<<grid_for(n, 256), 256, 0, s>>>((const float*)src, dst, n);
@@ -632,7 +675,7 @@ extern "C" VD_API vd_status vd_op_gn_stats_static(const void* x, int32_t dtype, 
         // the arrival counters live behind the records; they must be zero when the kernel starts
         unsigned int* counters = (unsigned int*)(partial + (size_t)kStaticGnMaxBatchTimesGroups * kGnMaxChunks * 2);
         e = cudaMemsetAsync(counters, 0, kStaticGnCounters * sizeof(unsigned int), (cudaStream_t)cuda_stream);
-        GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial, counters};
+        GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, partial, counters, nullptr};
         if (e == cudaSuccess) e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
     }
     if (e != cudaSuccess) {

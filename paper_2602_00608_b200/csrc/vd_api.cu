@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <map>
 #include <string>
 #include <vector>
 
@@ -28,6 +29,22 @@ struct Step {
     bool has_residual;
 };
 
+// A tensor-core convolution whose output only ever meets a GroupNorm, another convolution's residual add or the
+// fused shortcut leaves its bias out (its epilogue warps pace the narrow layers, and the additions are 40 of their
+// 70 instructions per pass).  The tensor then stands for "stored value + pending[c]", and the per-channel vector
+// `pending` is accounted for downstream: the statistics pass adds it on the fly and folds it into `shift`, a residual add
+// carries it along, the fused 1x1 shortcut contributes W * pending, and a convolution that reads the tensor without a
+// normalisation gets it as a unit-scale prologue.  The vectors depend on the weights alone: computed once in vd_create.
+constexpr size_t kNone = (size_t)-1;
+struct FoldJob {             // out[c] = in[c] + b[c] + b2[c] + sum_k w2[c][k] * pin[k]   (absent terms: kNone)
+    size_t out_off, in_off, b_off, b2_off, w2_off, pin_off;
+    int Cin2, Cout;
+};
+struct FillJob {             // dst[n][c] = src[c] (src kNone: 1.0) for n < B
+    size_t dst_off, src_off;
+    int C, B;
+};
+
 struct WeightJob {           // repack work done once in vd_create
     std::string name;        // source tensor
     int kind;                // 0 conv weight (packed), 1 vector -> fp32, 2 matrix [Cout][Cin] -> fp32 (same layout)
@@ -51,6 +68,8 @@ struct vd_handle_s {
     size_t ws_bytes = 0;
     std::vector<Step> steps;
     std::vector<WeightJob> jobs;
+    std::vector<FoldJob> folds;          // run once after the weight jobs, in order
+    std::vector<FillJob> fills;          // then these
     std::vector<size_t> guards;          // offsets of the guard regions (VD_FLAG_CANARY)
     std::string err;
     int stop_after = -1;
@@ -158,7 +177,8 @@ class Planner {
         s.kind = VD_STEP_GN_STATS;
         s.gn = GnArgs{ptr<void>(x_off), dtype, 0, H * W, C, cfg_.norm_groups, cfg_.norm_eps, ptr<float>(g_off),
                       ptr<float>(b_off), ptr<float>(scale_off_), ptr<float>(shift_off_), ptr<float>(partial_off_),
-                      ptr<unsigned int>(partial_off_ + gn_partial_bytes(cfg_.max_batch, cfg_.norm_groups))};
+                      ptr<unsigned int>(partial_off_ + gn_partial_bytes(cfg_.max_batch, cfg_.norm_groups)),
+                      pending(x_off) != kNone ? ptr<float>(pending(x_off)) : nullptr};
         fill_info(s, name, 0, C, C, 0, 0, H, W, C, VD_F32, 0, -1);
         s.info.launches = 1;
         s.info.bytes_per_frame = (double)H * W * C * elt(dtype);
@@ -208,6 +228,41 @@ class Planner {
             a.w2 = ptr<void>(w2_off);
             a.bias2 = ptr<float>(b2_off);
         }
+        // ---- pending biases (see FoldJob)
+        const bool want_defer = defer_;
+        defer_ = false;
+        const size_t pin_x = pending(x_off);
+        const size_t pres = residual_off >= 0 ? pending((size_t)residual_off) : kNone;
+        const size_t px2 = !shortcut_name.empty() ? pending(x2_off) : kNone;
+        if (!prologue && pin_x != kNone) {       // no normalisation in front: the pending bias enters as x * 1 + pending
+            if (ones_off_ == kNone) {
+                ones_off_ = alloc((size_t)cfg_.max_batch * max_c_ * 4);
+                h_->fills.push_back({ones_off_, kNone, max_c_ * cfg_.max_batch, 1});
+            }
+            const size_t sh = alloc((size_t)cfg_.max_batch * Cin * 4);
+            h_->fills.push_back({sh, pin_x, Cin, cfg_.max_batch});
+            a.scale = ptr<float>(ones_off_);
+            a.shift = ptr<float>(sh);
+        }
+        const size_t b2_off = a.bias2 ? (size_t)((const char*)a.bias2 - base_) : kNone;
+        const size_t w2_off = a.w2 ? (size_t)((const char*)a.w2 - base_) : kNone;
+        if (!y_is_frames) {
+            if (tc && want_defer && !(cfg_.flags & VD_FLAG_FUSED_STATS)) {
+                const size_t v = alloc((size_t)Cout * 4);
+                h_->folds.push_back({v, pres, cw.b_off, b2_off, px2 != kNone ? w2_off : kNone, px2, Cin2, Cout});
+                a.bias = nullptr;
+                a.bias2 = nullptr;
+                pending_[y_off] = v;
+            } else {
+                if (px2 != kNone) {               // the shortcut's share of its input's pending bias joins the shortcut bias
+                    const size_t v2 = alloc((size_t)Cout * 4);
+                    h_->folds.push_back({v2, kNone, kNone, b2_off, w2_off, px2, Cin2, Cout});
+                    a.bias2 = ptr<float>(v2);
+                }
+                if (pres != kNone) pending_[y_off] = pres;      // accumulated in place: what was pending stays pending
+                else pending_.erase(y_off);
+            }
+        }
         s.conv = a;
         s.use_tc = tc;
         s.has_residual = residual_off >= 0;
@@ -220,6 +275,7 @@ class Planner {
         s.info.weight_bytes = (double)ksize * ksize * Cin * Cout * elt(cfg_.dtype);
         s.info.has_residual = residual_off >= 0;
         s.info.phase_collapsed = phase ? 1 : 0;
+        if (!y_is_frames && pending(y_off) != kNone) s.info.out_pending_offset = (int64_t)pending(y_off);
         if (!shortcut_name.empty()) {
             s.info.c_in2 = Cin2;
             s.info.flops_per_frame += 2.0 * Cin2 * (double)Cout * P;
@@ -237,28 +293,33 @@ class Planner {
         s.info.c_in = cin; s.info.c_out = cout; s.info.ksize = ksize; s.info.upsample = up;
         s.info.out_h = H; s.info.out_w = W; s.info.out_channels = oc; s.info.out_dtype = odt;
         s.info.out_nchw = nchw; s.info.out_offset = off;
+        s.info.out_pending_offset = -1;
     }
 
     // x -> shortcut(x) + conv2(silu(gn2(conv1(silu(gn1(x))))))
     void resblock(const std::string& p, int Cin, int Cout, int H, int W) {
         const size_t x = xs_[cur_x_], y = xs_[cur_x_ ^ 1];
         add_gn(p + ".norm1", x, VD_F32, H, W, Cin, p + ".norm1");
+        defer_ = true;
         add_conv(p + ".conv1", {p + ".conv1"}, Cout, x, VD_F32, H, W, Cin, 3, false, true, true, -1, hbuf_, act_dtype(),
                  false, false);
         add_gn(p + ".norm2", hbuf_, act_dtype(), H, W, Cout, p + ".norm2");
         if (Cin == Cout) {
             // identity skip: conv2 accumulates into the residual stream in place (x += conv2(...))
+            defer_ = true;
             add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, (long)x, x,
                      VD_F32, false, false);
             return;
         }
         const bool fuse = bf16() && !(cfg_.flags & VD_FLAG_FORCE_SIMT) && Cout % 128 == 0 && Cin % 32 == 0;
         if (fuse) {      // the 1x1 shortcut rides along as extra K of conv2: no tensor of its own
+            defer_ = true;
             add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, -1, y,
                      VD_F32, false, false, p + ".shortcut", x, Cin);
         } else {
             add_conv(p + ".shortcut", {p + ".shortcut"}, Cout, x, VD_F32, H, W, Cin, 1, false, false, false, -1, y, VD_F32,
                      false, false);
+            defer_ = true;
             add_conv(p + ".conv2", {p + ".conv2"}, Cout, hbuf_, act_dtype(), H, W, Cout, 3, false, true, true, (long)y, y,
                      VD_F32, false, false);
         }
@@ -282,11 +343,13 @@ class Planner {
         s.info.flops_per_frame = 4.0 * T * T * C;
         s.info.bytes_per_frame = 4.0 * T * C * es;
         h_->steps.push_back(s);
+        defer_ = true;
         add_conv(p + ".o", {p + ".o"}, C, attno_, act_dtype(), H, W, C, 1, false, false, false, (long)x, x, VD_F32,
                  false, false);          // x += Wo o + bo, in place
     }
 
     void upconv(const std::string& p, int Cin, int Cout, int Hs, int Ws) {
+        defer_ = true;
         add_conv(p, {p}, Cout, xs_[cur_x_], VD_F32, Hs, Ws, Cin, 3, true, false, false, -1, xs_[cur_x_ ^ 1], VD_F32,
                  false, false);
         cur_x_ ^= 1;
@@ -325,6 +388,7 @@ class Planner {
             }
         }
         const int ae = elt(act_dtype());
+        max_c_ = (int)max_c;
         h_->status_off = alloc(256);
         for (int i = 0; i < 2; ++i) {
             scale_buf_[i] = alloc((size_t)B * max_c * 4);
@@ -413,6 +477,11 @@ class Planner {
     const vd_config& cfg_;
     size_t cur_ = 0;
     size_t stat_off_ = 0;
+    std::map<size_t, size_t> pending_;   // tensor offset -> offset of its pending-bias vector
+    size_t pending(size_t off) const { auto it = pending_.find(off); return it == pending_.end() ? kNone : it->second; }
+    bool defer_ = false;                 // set by the caller of add_conv: this layer's bias may be left pending
+    size_t ones_off_ = kNone;
+    int max_c_ = 0;
     size_t scale_off_ = 0, shift_off_ = 0, partial_off_ = 0, zbuf_ = 0, hbuf_ = 0, qkv_ = 0, attno_ = 0, vt_ = 0;
     size_t xs_[2] = {0, 0};
     size_t scale_buf_[2] = {0, 0}, shift_buf_[2] = {0, 0};
@@ -610,6 +679,15 @@ vd_status vd_create(const vd_config* cfg, const vd_tensor* weights, int32_t n_we
             e = launch_pack_weight_simt(t->dptr, t->dtype, (float*)(h->ws + j.dst_off), j.Cout, j.Cin, j.taps, j.cout_total, j.cout_offset, s);
         }
         if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, j.name.c_str()); }
+    }
+    auto at = [&](size_t off) -> float* { return off == kNone ? nullptr : (float*)(h->ws + off); };
+    for (const FoldJob& f : h->folds) {
+        e = launch_fold_bias(at(f.out_off), at(f.in_off), at(f.b_off), at(f.b2_off), at(f.w2_off), at(f.pin_off), f.Cin2, f.Cout, s);
+        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "bias fold"); }
+    }
+    for (const FillJob& f : h->fills) {
+        e = launch_fill_rows(at(f.dst_off), at(f.src_off), f.C, f.B, s);
+        if (e != cudaSuccess) { delete h; return cuda_fail(nullptr, e, "bias rows"); }
     }
     for (Step& st : h->steps) {
         if (st.kind == VD_STEP_CONV && st.use_tc) {
@@ -947,8 +1025,8 @@ size_t vd_gn_scratch_bytes(int32_t batch, int32_t groups) {
 }
 
 vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h, int32_t w, int32_t c, int32_t groups,
-                         float eps, const float* gamma, const float* beta, float* scale, float* shift, void* scratch,
-                         void* cuda_stream) {
+                         float eps, const float* gamma, const float* beta, const float* offset, float* scale, float* shift,
+                         void* scratch, void* cuda_stream) {
     if (!x || !gamma || !beta || !scale || !shift || !scratch) return fail(nullptr, VD_ERR_INVALID_ARG, "NULL pointer");
     if (dtype != VD_F32 && dtype != VD_BF16) return fail(nullptr, VD_ERR_INVALID_ARG, "bad dtype");
     if (batch < 0 || h < 1 || w < 1 || c < 1 || groups < 1 || c % groups != 0 || (c / groups) % 4 != 0 || c > 1024)
@@ -957,7 +1035,7 @@ vd_status vd_op_gn_stats(const void* x, int32_t dtype, int32_t batch, int32_t h,
         return fail(nullptr, VD_ERR_INVALID_ARG, "tensor too large (h*w must fit 31 bits, batch*h*w*c 40 bits)");
     if (batch == 0) return VD_OK;
     unsigned int* counters = (unsigned int*)((char*)scratch + gn_partial_bytes(batch, groups));
-    GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch, counters};
+    GnArgs a{x, dtype, batch, h * w, c, groups, eps, gamma, beta, scale, shift, (float*)scratch, counters, offset};
     cudaError_t e = cudaMemsetAsync(counters, 0, (size_t)batch * sizeof(unsigned int), (cudaStream_t)cuda_stream);
     if (e == cudaSuccess) e = launch_gn_stats(a, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? VD_OK : cuda_fail(nullptr, e, "vd_op_gn_stats");

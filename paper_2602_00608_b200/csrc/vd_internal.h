@@ -63,6 +63,8 @@ struct GnArgs {
     float* shift;           // [B,C]
     float* partial;         // [B, kGnMaxChunks, G, 2] scratch
     unsigned int* counters; // [B] arrival counters, zero before the launch; the kernel leaves them zero
+    const float* offset;    // [C] or null: the statistics are those of x + offset[c] (a bias the tensor's producer
+                            // left out), and shift takes scale * offset in, so scale * x + shift normalises x + offset
 };
 constexpr int kGnMaxChunks = 296;      // two blocks per SM on a 148-SM device
 // bytes of the partial records / of the whole scratch (records, then the arrival counters)
@@ -105,6 +107,11 @@ cudaError_t launch_pack_weight_simt(const void* w, int w_dtype, float* packed, i
                                     int cout_total, int cout_offset, cudaStream_t s);
 // any vector of dtype -> fp32
 cudaError_t launch_to_f32(const void* src, int dtype, float* dst, int64_t n, cudaStream_t s);
+// out[c] = in[c] + b[c] + b2[c] + sum_k w2[c][k] * pin[k], c < Cout (absent terms: null pointers)
+cudaError_t launch_fold_bias(float* out, const float* in, const float* b, const float* b2, const float* w2, const float* pin,
+                             int Cin2, int Cout, cudaStream_t s);
+// dst[n][c] = src[c] (src null: 1.0), n < B
+cudaError_t launch_fill_rows(float* dst, const float* src, int C, int B, cudaStream_t s);
 
 // ---- tcgen05 kernels (conv_tc.cu, attn_tc.cu)
 bool conv_tc_supported(const ConvArgs& a);

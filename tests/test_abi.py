@@ -37,7 +37,7 @@ def test_struct_sizes_match_the_header_layout(vd):
     assert ctypes.sizeof(vd.VdConfig) == 44
     assert ctypes.sizeof(vd.VdTensor) == 56
     assert ctypes.sizeof(vd.VdConvDesc) == 56
-    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 24
+    assert ctypes.sizeof(vd.VdStepInfo) == 64 + 12 * 4 + 8 + 3 * 8 + 24 + 8
 
 
 def test_query_workspace_is_host_only_and_scales_with_batch(vd):
@@ -87,7 +87,7 @@ def test_null_arguments_are_rejected_without_a_device(vd):
     assert l.vd_get_status(None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_num_steps(None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_op_conv2d(None, None, None, None, None, None, None, None, None) == vd.VD_ERR_INVALID_ARG
-    assert l.vd_op_gn_stats(None, 0, 1, 1, 1, 4, 1, 1e-6, None, None, None, None, None, None) == vd.VD_ERR_INVALID_ARG
+    assert l.vd_op_gn_stats(None, 0, 1, 1, 1, 4, 1, 1e-6, None, None, None, None, None, None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_op_attention(None, None, None, None, 0, 1, 1, 32, 32, 32, 1.0, 0, None, None) == vd.VD_ERR_INVALID_ARG
     assert l.vd_gn_scratch_bytes(0, 32) == 0
     assert b"NULL" in l.vd_last_error(None) or l.vd_last_error(None)

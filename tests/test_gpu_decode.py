@@ -161,12 +161,14 @@ def test_sdvae_bf16_degenerate_and_odd_sizes(env, h, w, b):
     dec, got, wts = _decode(env, wl, z)
     dec2, got2, _ = _decode(env, wl, z, flags=vd.VD_FLAG_FORCE_SIMT)
     assert got.shape == (b, 3, 8 * h, 8 * w)
-    d = got.float() - got2.float()
-    assert float(d.norm() / got2.float().norm()) <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
     if h * w <= 20:
         want = ref.decode(wl.arch, wts, z, wl.groups, wl.eps)
-        g = got.float().cpu().numpy()
-        assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+        for gg in (got, got2):
+            g = gg.float().cpu().numpy()
+            assert rel_l2(g, want) <= BF16_REL_L2 and max_abs(g, want) <= BF16_MAX_ABS
+    # two paths that each meet the bound against the exact result differ by at most twice the bound
+    d = got.float() - got2.float()
+    assert float(d.norm() / got2.float().norm()) <= 2 * BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
     dec.check_status()
 
 
