@@ -122,6 +122,27 @@ def test_gn_stats_match_two_pass_oracle(env, B, H, W, C, G, bf16):
         np.testing.assert_allclose(sh, wsh, rtol=2e-5, atol=2e-5)
 
 
+@pytest.mark.parametrize("B,H,W,C,G,bf16", [(2, 17, 23, 64, 8, False), (1, 31, 45, 256, 32, True), (1, 9, 5, 128, 32, False)])
+def test_gn_stats_with_a_per_channel_offset(env, B, H, W, C, G, bf16):
+    """scale * x + shift must normalise x + offset[c] (a bias the tensor's producer left out): against the
+    oracle's statistics of the shifted tensor."""
+    torch, ref, vd, synth = env
+    r = _rng(31)
+    x = r.standard_normal((B, C, H, W)).astype(np.float32) * 1.3 + 0.2
+    if bf16:
+        x = synth.round_to_bf16(x)
+    off = r.uniform(-2.0, 2.0, C).astype(np.float32)
+    gamma = r.uniform(0.9, 1.1, C).astype(np.float32)
+    beta = r.uniform(-0.1, 0.1, C).astype(np.float32)
+    want, _, _ = ref.groupnorm(x + off[None, :, None, None], gamma, beta, G, 1e-6, return_stats=True)
+    sc, sh = vd.op_gn_stats(util.nchw_to_dev_nhwc(x, torch.bfloat16 if bf16 else torch.float32),
+                            torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda(), G, 1e-6,
+                            offset=torch.from_numpy(off).cuda())
+    torch.cuda.synchronize()
+    got = x * sc.cpu().numpy()[:, :, None, None] + sh.cpu().numpy()[:, :, None, None]
+    assert rel_l2(got, want) <= 2e-5
+
+
 def test_gn_stats_survive_a_large_common_offset(env):
     # mean/std = 300: a plain sum-of-squares in fp32 would lose the variance
     sc, sh, wsc, wsh = _gn_case(env, 22, 1, 40, 40, 128, 32, False, offset=300.0)
