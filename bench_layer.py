@@ -40,13 +40,14 @@ def main():
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
     ap.add_argument("--impl", type=int, default=vd.VD_IMPL_TC)
+    ap.add_argument("--no-bias", action="store_true", help="no bias in the epilogue (the build the decoder runs where a layer's bias is pending)")
     a = ap.parse_args()
 
     g = torch.Generator(device="cuda").manual_seed(1)
     in_dt = torch.float32 if a.in_f32 else torch.bfloat16
     x = torch.randn((a.batch, a.h, a.w, a.cin), generator=g, device="cuda", dtype=torch.float32).to(in_dt)
     wt = (torch.rand((a.cout, a.cin, a.k, a.k), generator=g, device="cuda") - 0.5).to(torch.bfloat16)
-    bias = torch.zeros(a.cout, device="cuda")
+    bias = None if a.no_bias else torch.zeros(a.cout, device="cuda")   # None: the build the decoder runs where the bias is pending
     oh, ow = (2 * a.h, 2 * a.w) if a.upsample else (a.h, a.w)
     res = torch.randn((a.batch, oh, ow, a.cout), generator=g, device="cuda") if a.residual else None
     scale = torch.ones((a.batch, a.cin), device="cuda") if a.prologue else None
