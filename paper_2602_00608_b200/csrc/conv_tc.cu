@@ -337,7 +337,8 @@ __device__ void stat_finalize(const ConvArgs& a, int tid, void* smem_scratch) {
 // off, the extra live values cost the bf16-output kernels 1.4 % of a decode in spills)
 // BIAS: the epilogue adds the bias (a build without it for the layers whose bias is accounted for downstream: the
 // additions and the bias loads are more than half of a pass's instructions)
-template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false, bool BIAS = true>
+// X2: the layer has a second input (the fused 1x1 shortcut); the other builds carry none of its code
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
@@ -363,7 +364,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     // fp32 tile (16 x 8 pixels x 32 channels = 128 rows of 128 bytes) straight into an operand stage, the weights
     // come as fp32 too, and the products are tcgen05.mma kind::tf32 (K = 8) into the same accumulator.  Operands
     // keep 10 significant bits instead of bf16's 8; the tensor time of these chunks doubles, the producers' is gone.
-    const int kchunks2 = a.x2 ? (a.Cin2 >> 5) : 0;
+    const int kchunks2 = X2 ? (a.Cin2 >> 5) : 0;
     constexpr uint32_t SC_TILE_BYTES = TILE_H * TILE_W * 128;
     const int ktotal = kchunks + kchunks2;
     const int cout_pad = (a.Cout % 128 == 0) ? a.Cout : 16; // rows per tap in the packed weights
@@ -495,7 +496,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const uint32_t st_hi = st_lo + (uint32_t)(ITEMS * 16);
             // starts the copies of unit p; returns which of this thread's entries exist
             auto issue = [&](const Pos& p) -> uint32_t {
-                const bool second = p.kc >= kchunks;
+                const bool second = X2 && p.kc >= kchunks;
                 const int c0 = (second ? p.kc - kchunks : p.kc) * 64;
                 const bool centre_only = a.ksize == 1;
                 const Tile& tile = p.tile;
@@ -544,7 +545,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             };
             float sc[8], sh[8];
             auto load_affine = [&](const Pos& p) {               // GroupNorm scale/shift of the unit's channels
-                if (!prologue || p.kc >= kchunks) return;
+                if (!prologue || (X2 && p.kc >= kchunks)) return;
                 // channels of v[0..3] and v[4..7] (see load_raw); the tiles of an item lie in one frame
                 const int ca = p.kc * 64 + (IN_BF16 ? j * 8 : j * 4), cb = IN_BF16 ? ca + 4 : ca + 32;
                 const float* ps = a.scale + (size_t)p.tile.b * a.Cin;
@@ -571,7 +572,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const int cur_kc = nx.kc, cur_slot = nx.slot, cur_cnt = nx.cnt, cur_t = nx.t;
                 const bool cur_have = cur_cnt > 0;               // without a tile the CTA still follows the barriers
                 const uint32_t cur_vm = vm_next;
-                const bool second = cur_kc >= kchunks;
+                const bool second = X2 && cur_kc >= kchunks;
                 const bool pro = prologue;
                 constexpr bool in_bf16 = IN_BF16;
                 advance(nx);
@@ -636,7 +637,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             const int cnt = sched.mine(n);                   // 0: the peer of a two-CTA pair in an odd tail item
             const Tile tile0 = sched.get(cnt > 0 ? sched.index(t, 0) : t, BN);
             for (int kc = 0; kc < ktotal && ok; ++kc) {
-                const bool second = kc >= kchunks;             // a shortcut chunk: loaded by TMA, nothing to transform
+                const bool second = X2 && kc >= kchunks;       // a shortcut chunk: loaded by TMA, nothing to transform
                 const int c0 = kc * 64;
                 const bool centre_only = a.ksize == 1;
                 const bool pro = prologue && !second;
@@ -843,7 +844,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     if (has_bias && tl.n0 != bias_n0) {       // (re)load bias (+ shortcut bias) of this channel block
                         __syncwarp();
                         for (int i = lane; i < BN; i += 32)
-                            wbias[i] = (a.bias ? __ldg(a.bias + tl.n0 + i) : 0.f) + (a.bias2 ? __ldg(a.bias2 + tl.n0 + i) : 0.f);
+                            wbias[i] = (a.bias ? __ldg(a.bias + tl.n0 + i) : 0.f) + ((X2 && a.bias2) ? __ldg(a.bias2 + tl.n0 + i) : 0.f);
                         bias_n0 = tl.n0;
                         __syncwarp();
                     }
@@ -968,7 +969,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const Tile tl = sched.get(t, BN);
                 if constexpr (PH) break;                 // the phase form streams its weights in PhaseSched order, below
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
-                    const bool second = kc >= kchunks;
+                    const bool second = X2 && kc >= kchunks;
                     const int ntap = second ? 1 : taps;
                     for (int tap = 0; tap < ntap; ++tap) {
                         if (stage % Cfg::B_GROUP == 0) {     // stages come back in groups (see the MMA thread)
@@ -1129,8 +1130,8 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                         const bool centre = a.ksize == 1;                        // single centre tap
                         wait_on(smem_u32(&bars->a_full[as]), aph);
                         uint32_t a_row = a_lo0 + as * (A_STAGE_BYTES >> 4);
-                        if (kc >= kchunks) {
-                            if constexpr (CG == 1) shortcut_step(two_c, td, a_row);       // (always after the main chunks: accumulates)
+                        if (X2 && kc >= kchunks) {
+                            if constexpr (CG == 1 && X2) shortcut_step(two_c, td, a_row);       // (always after the main chunks: accumulates)
                         } else if (!centre) {
 #pragma unroll 1
                             for (int ky = 0; ky < 3; ++ky) {
@@ -1224,7 +1225,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const uint32_t td = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
                 uint32_t acc = 0;                             // the first MMA of an item overwrites the accumulator
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
-                    const bool centre = kc >= kchunks || a.ksize == 1;       // single centre tap
+                    const bool centre = (X2 && kc >= kchunks) || a.ksize == 1;       // single centre tap
                     const int ntap = centre ? 1 : 9;
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag));
                     if (!ok) break;
@@ -1438,9 +1439,9 @@ cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, 
     return cudaSuccess;
 }
 
-template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false, bool BIAS = true>
+template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS, BIAS>;
+    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS, BIAS, X2>;
     constexpr int SMEM = TileCfg<BN, CG, PH, IB>::SMEM_TOTAL;
     static KernelState state = {};
     int pairs = 0, sms = 0;
@@ -1502,7 +1503,7 @@ bool conv_tc_supported(const ConvArgs& a) {
     if (a.Cin % 64 != 0 || a.Cin < 64) return false;
     if (!a.bf16_operands) return false;
     if (a.ksize != 1 && a.ksize != 3) return false;
-    if (a.x2 && (a.Cin2 % 32 != 0 || a.Cin2 < 32 || a.upsample)) return false;
+    if (a.x2 && (a.Cin2 % 32 != 0 || a.Cin2 < 32 || a.upsample || a.in_dtype != VD_BF16 || a.out_dtype != VD_F32 || a.Cout % 128 != 0)) return false;
     if (a.upsample == 2)     // phase-collapsed form: 3x3, 128-channel blocks, plain NHWC store
         return a.ksize == 3 && a.Cout % 128 == 0 && !a.out_nchw && !a.residual && !a.x2;
     if (a.Cout % 128 == 0) return !a.out_nchw && !a.out_u8;
@@ -1654,6 +1655,10 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
     }
     if (plan.bn == 16) {
         return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
+    }
+    if (a.x2) {                // fused shortcut: bf16 intra-block input, fp32 output, one CTA per tile (conv_tc_supported)
+        if (plan.bn == 256) return hb ? launch_one<256, true, 0, 1, false, false, true, true>(a, plan, status, s) : launch_one<256, true, 0, 1, false, false, false, true>(a, plan, status, s);
+        return hb ? launch_one<128, true, 0, 1, false, false, true, true>(a, plan, status, s) : launch_one<128, true, 0, 1, false, false, false, true>(a, plan, status, s);
     }
 #define VD_CONV_CASE(BN_, CG_, PH_)                                                                                         \
     do {                                                                                                                    \
