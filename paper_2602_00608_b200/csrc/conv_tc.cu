@@ -338,7 +338,8 @@ __device__ void stat_finalize(const ConvArgs& a, int tid, void* smem_scratch) {
 // BIAS: the epilogue adds the bias (a build without it for the layers whose bias is accounted for downstream: the
 // additions and the bias loads are more than half of a pass's instructions)
 // X2: the layer has a second input (the fused 1x1 shortcut); the other builds carry none of its code
-template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false>
+// KS: kernel size, 3 or 1 (the 1x1 layers take the centre view of the halo tile only)
+template <int BN, bool IN_BF16, int OUT_MODE, int CG = 1, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false, int KS = 3>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2,
                const __grid_constant__ CUtensorMap tmap_y, const __grid_constant__ CUtensorMap tmap_x2, unsigned int* status) {
@@ -357,7 +358,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int taps = a.ksize * a.ksize;
+    constexpr int taps = KS * KS;
     const int kchunks = a.Cin >> 6;
     // Extra K: the 1x1 shortcut on a second input (fp32, at the output resolution), in sub-chunks of 32 channels.
     // It needs no halo and no transform, so it does not go through the producers: a bulk tensor load puts the
@@ -498,7 +499,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             auto issue = [&](const Pos& p) -> uint32_t {
                 const bool second = X2 && p.kc >= kchunks;
                 const int c0 = (second ? p.kc - kchunks : p.kc) * 64;
-                const bool centre_only = a.ksize == 1;
+                constexpr bool centre_only = KS == 1;
                 const Tile& tile = p.tile;
                 if (p.cnt == 0 || second) { cp_async_commit(); return 0u; }  // no tile of this CTA in the item, or a shortcut chunk (loaded by TMA): nothing to copy
                 uint32_t vm = 7u;
@@ -639,7 +640,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
             for (int kc = 0; kc < ktotal && ok; ++kc) {
                 const bool second = X2 && kc >= kchunks;       // a shortcut chunk: loaded by TMA, nothing to transform
                 const int c0 = kc * 64;
-                const bool centre_only = a.ksize == 1;
+                constexpr bool centre_only = KS == 1;
                 const bool pro = prologue && !second;
                 float sc[8], sh[8];
                 if (pro) {
@@ -1127,7 +1128,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                     uint32_t acc = 0;                         // the first MMA of an item overwrites the accumulator
 #pragma unroll 1
                     for (int kc = 0; kc < ktotal; ++kc) {
-                        const bool centre = a.ksize == 1;                        // single centre tap
+                        constexpr bool centre = KS == 1;                         // single centre tap
                         wait_on(smem_u32(&bars->a_full[as]), aph);
                         uint32_t a_row = a_lo0 + as * (A_STAGE_BYTES >> 4);
                         if (X2 && kc >= kchunks) {
@@ -1225,7 +1226,7 @@ conv_tc_kernel(const ConvArgs a, const __grid_constant__ CUtensorMap tmap, const
                 const uint32_t td = tmem_base + (uint32_t)(buf * PAIR * Cfg::ACC_COLS);
                 uint32_t acc = 0;                             // the first MMA of an item overwrites the accumulator
                 for (int kc = 0; kc < ktotal && ok; ++kc) {
-                    const bool centre = (X2 && kc >= kchunks) || a.ksize == 1;       // single centre tap
+                    const bool centre = (X2 && kc >= kchunks) || KS == 1;            // single centre tap
                     const int ntap = centre ? 1 : 9;
                     ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->a_full[as]), aph, abort_flag));
                     if (!ok) break;
@@ -1439,9 +1440,9 @@ cudaError_t kernel_state(K kern, int smem, int cg, KernelState& st, int* pairs, 
     return cudaSuccess;
 }
 
-template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false>
+template <int BN, bool IB, int OM, int CG, bool PH = false, bool STATS = false, bool BIAS = true, bool X2 = false, int KS = 3>
 cudaError_t launch_one(const ConvArgs& a, const ConvTcPlan& plan, unsigned int* status, cudaStream_t s) {
-    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS, BIAS, X2>;
+    auto kern = conv_tc_kernel<BN, IB, OM, CG, PH, STATS, BIAS, X2, KS>;
     constexpr int SMEM = TileCfg<BN, CG, PH, IB>::SMEM_TOTAL;
     static KernelState state = {};
     int pairs = 0, sms = 0;
@@ -1503,7 +1504,8 @@ bool conv_tc_supported(const ConvArgs& a) {
     if (a.Cin % 64 != 0 || a.Cin < 64) return false;
     if (!a.bf16_operands) return false;
     if (a.ksize != 1 && a.ksize != 3) return false;
-    if (a.x2 && (a.Cin2 % 32 != 0 || a.Cin2 < 32 || a.upsample || a.in_dtype != VD_BF16 || a.out_dtype != VD_F32 || a.Cout % 128 != 0)) return false;
+    if (a.ksize == 1 && (a.upsample || a.Cout % 128 != 0)) return false;       // 1x1: plain layers of 128-channel blocks
+    if (a.x2 && (a.Cin2 % 32 != 0 || a.Cin2 < 32 || a.upsample || a.ksize != 3 || a.in_dtype != VD_BF16 || a.out_dtype != VD_F32 || a.Cout % 128 != 0)) return false;
     if (a.upsample == 2)     // phase-collapsed form: 3x3, 128-channel blocks, plain NHWC store
         return a.ksize == 3 && a.Cout % 128 == 0 && !a.out_nchw && !a.residual && !a.x2;
     if (a.Cout % 128 == 0) return !a.out_nchw && !a.out_u8;
@@ -1648,29 +1650,36 @@ cudaError_t launch_conv_tc(const ConvArgs& a, const ConvTcPlan& plan, unsigned i
         return cudaErrorInvalidValue;
     const bool ib = a.in_dtype == VD_BF16, ob = a.out_dtype == VD_BF16;
     const bool hb = a.bias != nullptr || a.bias2 != nullptr;
+    const bool k1 = a.ksize == 1;
     if (a.stat_sum) {          // bf16 output with the statistics of the following GroupNorm (checked above)
         if (plan.bn == 256 && plan.cg == 2) return ib ? launch_one<256, true, 1, 2, false, true>(a, plan, status, s) : launch_one<256, false, 1, 2, false, true>(a, plan, status, s);
-        if (plan.bn == 256) return ib ? launch_one<256, true, 1, 1, false, true>(a, plan, status, s) : launch_one<256, false, 1, 1, false, true>(a, plan, status, s);
+        if (plan.bn == 256) {
+            if (k1) return ib ? launch_one<256, true, 1, 1, false, true, true, false, 1>(a, plan, status, s) : launch_one<256, false, 1, 1, false, true, true, false, 1>(a, plan, status, s);
+            return ib ? launch_one<256, true, 1, 1, false, true>(a, plan, status, s) : launch_one<256, false, 1, 1, false, true>(a, plan, status, s);
+        }
+        if (k1) return ib ? launch_one<128, true, 1, 1, false, true, true, false, 1>(a, plan, status, s) : launch_one<128, false, 1, 1, false, true, true, false, 1>(a, plan, status, s);
         return ib ? launch_one<128, true, 1, 1, false, true>(a, plan, status, s) : launch_one<128, false, 1, 1, false, true>(a, plan, status, s);
     }
     if (plan.bn == 16) {
+        if (k1) return cudaErrorInvalidValue;                  // the frame head is a 3x3 layer
         return ib ? launch_one<16, true, 2, 1>(a, plan, status, s) : launch_one<16, false, 2, 1>(a, plan, status, s);
     }
-    if (a.x2) {                // fused shortcut: bf16 intra-block input, fp32 output, one CTA per tile (conv_tc_supported)
+    if (a.x2) {                // fused shortcut: 3x3, bf16 intra-block input, fp32 output, one CTA per tile (conv_tc_supported)
         if (plan.bn == 256) return hb ? launch_one<256, true, 0, 1, false, false, true, true>(a, plan, status, s) : launch_one<256, true, 0, 1, false, false, false, true>(a, plan, status, s);
         return hb ? launch_one<128, true, 0, 1, false, false, true, true>(a, plan, status, s) : launch_one<128, true, 0, 1, false, false, false, true>(a, plan, status, s);
     }
-#define VD_CONV_CASE(BN_, CG_, PH_)                                                                                         \
+#define VD_CONV_CASE(BN_, CG_, PH_, KS_)                                                                                    \
     do {                                                                                                                    \
-        if (ib && ob) return hb ? launch_one<BN_, true, 1, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, true, 1, CG_, PH_, false, false>(a, plan, status, s);     \
-        if (ib && !ob) return hb ? launch_one<BN_, true, 0, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, true, 0, CG_, PH_, false, false>(a, plan, status, s);    \
-        if (!ib && ob) return hb ? launch_one<BN_, false, 1, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, false, 1, CG_, PH_, false, false>(a, plan, status, s);  \
-        return hb ? launch_one<BN_, false, 0, CG_, PH_, false, true>(a, plan, status, s) : launch_one<BN_, false, 0, CG_, PH_, false, false>(a, plan, status, s);                 \
+        if (ib && ob) return hb ? launch_one<BN_, true, 1, CG_, PH_, false, true, false, KS_>(a, plan, status, s) : launch_one<BN_, true, 1, CG_, PH_, false, false, false, KS_>(a, plan, status, s);     \
+        if (ib && !ob) return hb ? launch_one<BN_, true, 0, CG_, PH_, false, true, false, KS_>(a, plan, status, s) : launch_one<BN_, true, 0, CG_, PH_, false, false, false, KS_>(a, plan, status, s);    \
+        if (!ib && ob) return hb ? launch_one<BN_, false, 1, CG_, PH_, false, true, false, KS_>(a, plan, status, s) : launch_one<BN_, false, 1, CG_, PH_, false, false, false, KS_>(a, plan, status, s);  \
+        return hb ? launch_one<BN_, false, 0, CG_, PH_, false, true, false, KS_>(a, plan, status, s) : launch_one<BN_, false, 0, CG_, PH_, false, false, false, KS_>(a, plan, status, s);                 \
     } while (0)
-    if (plan.phase) VD_CONV_CASE(128, 2, true);
-    if (plan.bn == 256 && plan.cg == 2) VD_CONV_CASE(256, 2, false);
-    if (plan.bn == 256) VD_CONV_CASE(256, 1, false);
-    VD_CONV_CASE(128, 1, false);
+    if (plan.phase) VD_CONV_CASE(128, 2, true, 3);
+    if (plan.bn == 256 && plan.cg == 2) VD_CONV_CASE(256, 2, false, 3);          // (9-tap upsampling form: 3x3)
+    if (plan.bn == 256) { if (k1) VD_CONV_CASE(256, 1, false, 1); VD_CONV_CASE(256, 1, false, 3); }
+    if (k1) VD_CONV_CASE(128, 1, false, 1);
+    VD_CONV_CASE(128, 1, false, 3);
 #undef VD_CONV_CASE
 }
 
