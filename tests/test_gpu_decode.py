@@ -150,6 +150,22 @@ def test_full_size_configs_whole_frame_against_the_oracle(env, idx):
     assert r2 <= BF16_REL_L2 and float(d.abs().max()) <= 2 * BF16_MAX_ABS
 
 
+@pytest.mark.parametrize("flags_name", ["VD_FLAG_FUSED_STATS", "VD_FLAG_UPSAMPLE_9TAP"])
+def test_full_size_720x480_whole_frame_with_the_optional_forms(env, flags_name):
+    """The selectable forms of the same decoder at full size, every pixel against the stored oracle frame: GroupNorm
+    statistics taken in the convolutions' epilogues, and upsampling as nine taps on the 2x grid."""
+    torch, ref, vd, synth = env
+    gold = np.load(os.path.join(GOLDEN, "frame_cfg3_full.npz"))
+    wl = synth.WORKLOADS[3]
+    z = synth.workload_latents(wl)
+    dec, got, _ = _decode(env, wl, z, flags=getattr(vd, flags_name))
+    g = got[int(gold["index"])].float().cpu().numpy()
+    r, m = rel_l2(g, gold["frame"]), max_abs(g, gold["frame"])
+    print(f"whole-frame parity {wl.name} with {flags_name}: rel-L2 {r:.3e} max-abs {m:.3e}")
+    assert r <= BF16_REL_L2 and m <= BF16_MAX_ABS, (r, m)
+    dec.check_status()
+
+
 @pytest.mark.parametrize("h,w,b", [(1, 1, 1), (2, 3, 2), (5, 4, 3), (33, 47, 2)])
 def test_sdvae_bf16_degenerate_and_odd_sizes(env, h, w, b):
     """Latents smaller than one tile (every tile of every level ragged, most of each halo outside the image), and a
